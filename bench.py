@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the sampling-verification hot path (SpecHub + RRS + RRSw).
+
+One step = the whole hot path over one synthetic batch: for each of the three
+methods, the draft step, the verification of every tree node and the tree walk,
+all on one stream.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
+
+Timing: CUDA events on the launching stream, barrier + synchronize on both
+sides, max over ranks.  Inputs (several GB) are far larger than L2, so no flush
+is needed between steps.  Multi-GPU: every rank runs its own batch of the same
+shape (no collective on the data path), so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "tree-nodes verified/sec"
+UNIT = "nodes/s"
+METHODS = ("spechub", "rrs", "rrsw")
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--layout", default="dense", choices=["dense", "paper"],
+                    help="dense: every node verifies; paper: last-level nodes only draw the bonus token")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle timing leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def config_dict(cfg, layout, n_gpus):
+    return {
+        "workload": "%s: batch %d x %d-node binary tree, V=%d, %s logits, T=%g, layout=%s" % (
+            cfg.name, cfg.batch, cfg.nodes, cfg.vocab, cfg.dtype, cfg.temperature, layout),
+        "methods": list(METHODS),
+        "global_batch": cfg.batch * n_gpus,
+        "nodes": cfg.nodes,
+        "vocab": cfg.vocab,
+        "parallelism": "batch-sharded x%d, no collective" % n_gpus,
+        "l2": "inputs larger than L2 (%.2f GB per rank)" % (2 * cfg.rows * cfg.vocab * (2 if cfg.dtype == "bf16" else 4) / 1e9),
+    }
+
+
+# ---- the oracle leg (CPU baseline, and --impl reference) -----------------------------------------
+
+def oracle_sample(cfg, layout, seconds):
+    """Time the CPU oracle, as it stands, on whole sequences of the workload until about
+    `seconds` of work is done.  Returns (node verifications per second, description)."""
+    import oracle
+
+    oracle.build()
+    kind = workloads.paper_node_kind(cfg.nodes) if layout == "paper" else None
+    prior = workloads._prior(cfg)
+    done_nodes, spent, b = 0, 0.0, 0
+    while True:
+        lp, lq = workloads.host_sequence(cfg, b % cfg.batch, prior)
+        un = workloads.host_uniforms(cfg, [b % cfg.batch])
+        lp, lq = lp[None], lq[None]
+        t0 = time.perf_counter()
+        for m in METHODS:
+            d = oracle.draft_batch(m, lq, cfg.temperature, un)
+            out = oracle.verify_batch(m, lp, lq, cfg.temperature, d["tokens"], un, kind)
+            oracle.walk(out["accept_idx"], out["token"], cfg.levels, node_kind=kind)
+        spent += time.perf_counter() - t0
+        done_nodes += len(METHODS) * cfg.nodes
+        b += 1
+        if spent >= seconds or b >= cfg.batch:
+            break
+    return done_nodes / spent, "%d whole sequences (%d nodes each) x %d methods, %.1f s" % (
+        b, cfg.nodes, len(METHODS), spent), spent
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(0.5, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, args.layout, per_step / 4)
+    vals, times = [], []
+    for _ in range(args.steps):
+        v, desc, spent = oracle_sample(cfg, args.layout, per_step)
+        vals.append(v); times.append(spent)
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_dict(cfg, args.layout, 1),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": "each step: " + desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---- clocks ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            cmd = ["nvidia-smi", "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd += ["-i", self.uuid]
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(np.max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- the GPU arm -------------------------------------------------------------------------------------
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s)"
+
+
+def main():
+    args = parse()
+    cfg = workloads.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2411_05289_b200 as sh
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    sh.load_library()
+
+    # this rank's batch (same shape on every rank, its own seed)
+    from dataclasses import replace
+
+    rcfg = replace(cfg, seed=cfg.seed + 17 * rank)
+    tp, tq = workloads.device_logits(rcfg, device=dev)
+    un = workloads.device_uniforms(rcfg, device=dev)
+    B, N, V = tp.shape
+    tree = sh.Tree.heap(N, leaves_sample=(args.layout == "paper"), device=dev)
+    from paper_2411_05289_b200.binding import alloc_verify_outputs
+
+    outs = {m: alloc_verify_outputs(B, N, tree.levels, dev) for m in METHODS}
+    stream = torch.cuda.current_stream()
+    ev_pairs = []
+
+    def step(record=False):
+        for m in METHODS:
+            if m == "spechub":
+                d = sh.spechub_draft_sample(tq, un, tree, cfg.temperature)
+            else:
+                d = sh.rrs_draft_sample(tq, un, tree, m == "rrsw", cfg.temperature)
+            if record and m == "spechub":
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            if m == "spechub":
+                sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=outs[m])
+            else:
+                sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=outs[m])
+            if record and m == "spechub":
+                e1.record(stream)
+                ev_pairs.append((e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        pass
+    clk = ClockSampler(uuid)
+    if rank == 0:
+        clk.start()
+        time.sleep(0.3)
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(args.steps):
+        step(record=True)
+    t1.record(stream)
+    barrier()
+    ms = t0.elapsed_time(t1)
+    clocks = clk.stop() if rank == 0 else None
+    # the walk kernel is inside the recorded span; it is a few microseconds
+    verify_ms = float(np.mean([a.elapsed_time(b) for a, b in ev_pairs]))
+
+    # ---- end to end: host buffers in, host results out, through the public API ----
+    esz = 2 if cfg.dtype == "bf16" else 4
+    h_tp = torch.empty(tp.shape, dtype=tp.dtype, pin_memory=True); h_tp.copy_(tp)
+    h_tq = torch.empty(tq.shape, dtype=tq.dtype, pin_memory=True); h_tq.copy_(tq)
+    h_un = torch.empty(un.shape, dtype=un.dtype, pin_memory=True); h_un.copy_(un)
+    res_keys = ("n_accepted", "n_emitted", "path_tokens", "accept_idx", "token")
+    h_res = {m: {k: torch.empty(outs[m][k].shape, dtype=outs[m][k].dtype, pin_memory=True) for k in res_keys}
+             for m in METHODS}
+    h2d = (h_tp.numel() + h_tq.numel()) * esz + h_un.numel() * 4
+    d2h = sum(v.numel() * v.element_size() for m in METHODS for v in h_res[m].values())
+
+    def e2e_step():
+        tp.copy_(h_tp, non_blocking=True)
+        tq.copy_(h_tq, non_blocking=True)
+        un.copy_(h_un, non_blocking=True)
+        step()
+        for m in METHODS:
+            for k in res_keys:
+                h_res[m][k].copy_(outs[m][k], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    w0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - w0
+
+    tms = torch.tensor([ms, e2e_s * 1e3, verify_ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms, e2e_ms, verify_ms = [float(x) for x in tms.tolist()]
+
+    if rank == 0:
+        nodes_per_step = len(METHODS) * B * N * world
+        value = nodes_per_step * args.steps / (ms * 1e-3)
+        e2e_value = nodes_per_step * args.e2e_steps / (e2e_ms * 1e-3)
+        kind = workloads.paper_node_kind(N) if args.layout == "paper" else np.zeros(N, np.uint8)
+        n_leaf = int(kind.sum())
+        alg_bytes = B * ((N - n_leaf) * (2 * V * esz + 8 + 20 + 44) + n_leaf * (V * esz + 20 + 44))
+        peak, peak_src = measured_peak()
+        achieved = alg_bytes / (verify_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": config_dict(cfg, args.layout, world),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": args.e2e_steps},
+            "gpu_launches": 9 * args.steps,
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "spechub_verify_tree (verification kernel + walk)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / 8000.0,
+                         "traffic": None, "alg_bytes_per_launch": alg_bytes, "ms_per_launch": verify_ms},
+            "breakdown": {
+                "spechub_verify_nodes_per_s": B * N / (verify_ms * 1e-3),
+                "spechub_verify_vocab_elements_per_s": B * N * V / (verify_ms * 1e-3),
+                "step_vocab_elements_per_s": nodes_per_step * V * args.steps / (ms * 1e-3),
+            },
+        }
+        if not args.no_cpu_baseline and world == 1:
+            v, desc, _ = oracle_sample(cfg, args.layout, args.cpu_seconds)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,208 @@
+/*
+ * spechub.h -- C ABI of the sampling-verification step of multi-draft
+ * speculative decoding: SpecHub (k = 2) with Recursive Rejection Sampling
+ * with and without replacement (RRS, RRSw) as the comparison path
+ * (arXiv 2411.05289).
+ *
+ * Notation is the paper's (Section 2): p = target distribution, q = draft
+ * distribution over a vocabulary of size V; a = argmax q is the hub token
+ * (Section 4); each tree node carries k = 2 draft tokens (x1, x2), one per
+ * child.  Both distributions are given as logits and a temperature T:
+ * p = softmax(target_logits / T), q = softmax(draft_logits / T).
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, valid until
+ *     the work enqueued on `stream` has finished.  The descriptor itself is
+ *     read on the host during the call.  The library allocates nothing and
+ *     keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work and return without synchronising.
+ *   - Return value: SPECHUB_OK (0) when the work was enqueued; a negative
+ *     SPECHUB_ERR_* when an argument was rejected on the host (nothing was
+ *     launched) or a launch failed.  Nothing is printed, nothing throws.
+ *     batch = 0 is a valid empty call: it returns SPECHUB_OK without looking
+ *     at any data pointer.
+ *   - Per-row problems found on the device are reported as bits in the row's
+ *     `status` word and give the documented fallback output; kernels never
+ *     trap and wait only on hardware barriers.
+ *   - Layout: logits are [batch][nodes][vocab] with element strides
+ *     `stride_seq`, `stride_node` (rows are contiguous in the vocabulary).
+ *     Rows that start on a 16-byte boundary are read with 128-bit loads; other
+ *     rows are still read correctly, element by element.
+ *     uniforms are float [batch][nodes][5] = (u_d1, u_d2, r1, r2, u_res), each
+ *     in [0, 1): u_d1, u_d2 drive the two draft draws; r1, r2 the first and
+ *     second acceptance test performed at the node; u_res the residual (or
+ *     leaf) draw.  draft_tokens are int32 [batch][nodes][2]; per-node outputs
+ *     are [batch][nodes] (row-major), with 2 or 3 trailing entries where
+ *     stated.
+ *   - Sampling from a non-negative weight vector w with a uniform u always
+ *     means: the lowest token id j whose inclusive prefix sum over ascending
+ *     ids exceeds u * sum(w); zero-weight ids are never returned.
+ *   - An acceptance test with probability min(N/D, 1) is the strict test
+ *     r * D < N; D = 0 rejects.
+ */
+#ifndef SPECHUB_H_
+#define SPECHUB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECHUB_ABI_VERSION 1
+
+/* return codes */
+#define SPECHUB_OK 0
+#define SPECHUB_ERR_NULL (-1)        /* a required pointer is NULL                        */
+#define SPECHUB_ERR_VERSION (-2)     /* struct_size / version do not match this library   */
+#define SPECHUB_ERR_SHAPE (-3)       /* batch < 0, nodes < 1, vocab < 2, k != 2, levels < 1 */
+#define SPECHUB_ERR_DTYPE (-4)       /* dtype is not SPECHUB_F32 / SPECHUB_BF16            */
+#define SPECHUB_ERR_STRIDE (-5)      /* stride_node < vocab or stride_seq too small        */
+#define SPECHUB_ERR_TEMPERATURE (-6) /* temperature not a finite number > 0               */
+#define SPECHUB_ERR_WORKSPACE (-7)   /* workspace smaller than spechub_workspace_bytes()   */
+#define SPECHUB_ERR_LAUNCH (-8)      /* the CUDA runtime refused a launch                  */
+#define SPECHUB_ERR_METHOD (-9)      /* without_replacement is not 0 or 1                  */
+
+/* logits element type */
+#define SPECHUB_F32 0
+#define SPECHUB_BF16 1
+
+/* per-row status bits */
+#define SPECHUB_ST_NONFINITE 1u       /* NaN or +inf logit, or no finite logit: row output is -1 */
+#define SPECHUB_ST_TOKEN_RANGE 2u     /* draft token out of range / pair lacks the hub: output -1  */
+#define SPECHUB_ST_DEGENERATE_Q 4u    /* draft mass outside the excluded token is 0 (one-hot q)    */
+#define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
+#define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
+
+/* node kinds */
+#define SPECHUB_NODE_VERIFY 0 /* run the accept/reject tests on the node's two drafts         */
+#define SPECHUB_NODE_LEAF 1   /* no drafts below: draw the bonus token from p with u_res       */
+
+typedef struct spechub_desc {
+    uint32_t struct_size; /* sizeof(spechub_desc)                                            */
+    uint32_t version;     /* SPECHUB_ABI_VERSION                                             */
+    int32_t batch;        /* sequences B                                                     */
+    int32_t nodes;        /* tree nodes per sequence N, level order, node 0 = root           */
+    int32_t vocab;        /* V >= 2                                                          */
+    int32_t k;            /* drafts per node; must be 2 (Section 4)                          */
+    int32_t dtype;        /* SPECHUB_F32 or SPECHUB_BF16 logits                              */
+    int32_t levels;       /* longest root-to-leaf path in nodes; bounds the walk, row length
+                             of the path outputs                                             */
+    int64_t stride_seq;   /* elements between consecutive sequences of a logits tensor       */
+    int64_t stride_node;  /* elements between consecutive nodes                              */
+    float temperature;    /* T > 0, used when temperature_per_seq is NULL                    */
+    const float *temperature_per_seq; /* device [batch] or NULL                               */
+    const int32_t *child;   /* device [nodes][2]: node reached by accepting draft i, < 0 = none;
+                               NULL = complete binary tree in heap order, child i of n is 2n+1+i */
+    const uint8_t *node_kind; /* device [nodes]: SPECHUB_NODE_*; NULL = every node verifies    */
+    uint32_t flags;       /* reserved, must be 0                                             */
+} spechub_desc;
+
+/* Per-node outputs, each a device array [batch][nodes] (x trailing count).
+ * accept_idx and token are required; the others may be NULL. */
+typedef struct spechub_node_out {
+    int32_t *accept_idx; /* 0 / 1: child whose draft was accepted; -1: rejected, leaf or flagged */
+    int32_t *token;      /* token emitted at this node: accepted draft, residual or leaf draw;
+                            -1 on SPECHUB_ST_NONFINITE / SPECHUB_ST_TOKEN_RANGE                */
+    int32_t *hub;        /* a (SpecHub), -1 for RRS / RRSw and leaves                          */
+    float *beta;         /* [..][2] acceptance probability of test 1 / test 2 for this pair     */
+    float *rate;         /* [..][3] row masses: accept child 0, accept child 1, reject          */
+    uint32_t *status;    /* SPECHUB_ST_* bits                                                   */
+} spechub_node_out;
+
+/* Per-sequence outputs of the tree walk (Figure 2); any pointer may be NULL,
+ * and a NULL seq_out skips the walk. */
+typedef struct spechub_seq_out {
+    int32_t *n_accepted;  /* [batch] accepted draft tokens on the path                         */
+    int32_t *n_emitted;   /* [batch] tokens emitted this step (accepted + residual/bonus)       */
+    int32_t *path_nodes;  /* [batch][levels] visited nodes, padded with -1                      */
+    int32_t *path_tokens; /* [batch][levels] emitted tokens, padded with -1                     */
+} spechub_seq_out;
+
+/*
+ * Draft step of SpecHub (Section 4; Algorithm 3, "Sample draft tokens
+ * x1, x2 ~ Q").  For every node: a = argmax of the draft logits (lowest id on
+ * ties); (x1, x2) is drawn from the sparse joint distribution
+ *   Q(x, a) = q(x),   Q(a, x) = q(a) q(x) / (1 - q(a))   (x != a), 0 elsewhere:
+ * x1 is drawn from q with u_d1; if x1 != a then x2 = a, otherwise x2 is drawn
+ * with u_d2 from q restricted to ids != a.
+ *   draft_logits  [B][N][V] of desc->dtype        (in)
+ *   uniforms      [B][N][5]                       (in; entries 0 and 1 are used)
+ *   draft_tokens  [B][N][2]                       (out)
+ *   hub           [B][N]                          (out, may be NULL)
+ *   draft_prob    [B][N][2] = (q(a), Q(x1, x2))   (out, may be NULL)
+ *   status        [B][N]                          (out, may be NULL)
+ * A one-hot q (1 - q(a) = 0) yields (a, lowest id != a) with
+ * SPECHUB_ST_DEGENERATE_Q; a flagged NONFINITE row yields (-1, -1).
+ */
+int spechub_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                         int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
+                         void *stream);
+
+/*
+ * Draft step of RRS / RRSw (Algorithm 1, "Generate k samples ... independently
+ * or without replacement from q").  x1 is drawn from q with u_d1; x2 from q
+ * with u_d2 (without_replacement = 0) or from q with q(x1) set to 0
+ * (without_replacement = 1).  Arguments as above.
+ */
+int rrs_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                     int without_replacement, int32_t *draft_tokens, uint32_t *status, void *stream);
+
+/*
+ * Verification with SpecHub (Algorithm 3 with Algorithm 2, Appendix B.1; the
+ * closed-form transport of Section 4) of every node, then the tree walk
+ * (Figure 2).  With c = q(a) / (1 - q(a)) and, over ids y != a,
+ *   S1 = sum max(q - p, 0),  S2 = sum max(c q - max(p - q, 0), 0),
+ *   R  = sum max(max(p - q, 0) - c q, 0):
+ *   pair (x, a): accept x (child 0) iff r1 q(x) < p(x); else accept a (child 1)
+ *                iff r2 S1 < max(p(a) - S2, 0);
+ *   pair (a, x): accept x (child 1) iff r1 c q(x) < max(p(x) - q(x), 0); else
+ *                accept a (child 0) iff r2 S2 < p(a);
+ *   otherwise the token is drawn with u_res from the residual
+ *   max(max(p - q, 0) - c q, 0), which has no mass on a.
+ * rate = (sum min(p,q) + min(p(a), S2),
+ *         sum min(max(p-q,0), c q) + min(max(p(a) - S2, 0), S1),  R).
+ * A pair that does not contain the hub exactly once is flagged TOKEN_RANGE.
+ * Leaf nodes (desc->node_kind) read only target_logits.
+ *   target_logits, draft_logits [B][N][V]   (in)
+ *   draft_tokens [B][N][2], uniforms [B][N][5] (in; entries 2, 3, 4 are used)
+ *   node_out (required), seq_out (may be NULL)
+ *   workspace: device scratch of at least spechub_workspace_bytes(desc) bytes;
+ *   may be NULL when that is 0.
+ */
+int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
+                        const void *draft_logits, const int32_t *draft_tokens,
+                        const float *uniforms, const spechub_node_out *node_out,
+                        const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                        void *stream);
+
+/*
+ * Verification with Recursive Rejection Sampling (Algorithm 1) of every node,
+ * then the tree walk.  With A1 = sum max(p - q, 0) and q1 = q (RRS) or q with
+ * q(x1) zeroed and renormalised (RRSw):
+ *   accept x1 (child 0) iff r1 q(x1) < p(x1); else accept x2 (child 1) iff
+ *   r2 A1 q1(x2) < max(p(x2) - q(x2), 0); otherwise draw with u_res from
+ *   max(max(p - q, 0) - A1 q1, 0).
+ * rate = (sum min(p,q), A1 - W2, W2), W2 the mass of that last residual (for
+ * RRSw the last two are for the given x1).  hub is written as -1.
+ */
+int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                    const int32_t *draft_tokens, const float *uniforms, int without_replacement,
+                    const spechub_node_out *node_out, const spechub_seq_out *seq_out,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Scratch bytes the two verify calls need for this descriptor (0 is possible). */
+size_t spechub_workspace_bytes(const spechub_desc *desc);
+
+/* Static, NUL-terminated description of a return code. */
+const char *spechub_status_string(int code);
+
+/* SPECHUB_ABI_VERSION the library was built with. */
+int spechub_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECHUB_H_ */

@@ -32,6 +32,7 @@ NODE_DTYPE = np.dtype(
         ("beta", np.float64, (2,)),
         ("rate", np.float64, (3,)),
         ("margin", np.float64, (3,)),
+        ("cond", np.float64, (2,)),
         ("accept_idx", np.int32),
         ("token", np.int32),
         ("hub", np.int32),

@@ -141,6 +141,10 @@ typedef struct {
     double beta[2];    /* acceptance probability min(N/D,1) of test 1 / test 2 for this pair  */
     double rate[3];    /* row-level masses: accept child 0, accept child 1, reject              */
     double margin[3];  /* |r1 - N1/D1|, |r2 - N2/D2| (inf if not performed), residual-draw margin */
+    double cond[2];    /* conditioning of N/D for test 1 / test 2: (|N| + beta |D|) / D, where |.|
+                          is the sum of the absolute values of the terms the quantity is formed
+                          from; a relative error eps in every p(y), q(y) moves N/D by at most
+                          eps * cond.  Used only by the parity checker to size its tolerance. */
     int32_t accept_idx; /* 0 / 1 = accepted child, -1 = rejected (token is the residual draw)  */
     int32_t token;      /* emitted token of this node                                          */
     int32_t hub;        /* a (SpecHub) or -1                                                   */
@@ -154,9 +158,10 @@ static void node_clear(orc_node *o) {
 }
 
 /* One strict multiplicative acceptance test: accept iff D > 0 and r*D < N. */
-static int accept_test(double r, double N, double D, double *beta, double *margin, int performed,
-                       uint32_t *status) {
+static int accept_test(double r, double N, double D, double normN, double normD, double *beta,
+                       double *cond, double *margin, int performed, uint32_t *status) {
     *beta = (D > 0.0) ? dmin(N / D, 1.0) : 0.0;
+    *cond = (D > 0.0) ? (normN + *beta * normD) / D : 0.0;
     if (!performed) return 0;
     if (!(D > 0.0)) { *status |= ORC_ZERO_MASS_DRAFT; *margin = INFINITY; return 0; }
     *margin = fabs(r - N / D);
@@ -266,8 +271,11 @@ void orc_spechub_verify(const double *p, const double *q, int V, int a, int x1, 
     p2[a] = 0.0;                               /* residual carries no hub mass */
 
     nsum s1, s2, m1, m2, rr; ns_init(&s1); ns_init(&s2); ns_init(&m1); ns_init(&m2); ns_init(&rr);
+    double nS1 = 0.0, nS2 = 0.0;               /* term magnitudes, for cond[] only */
     for (int y = 0; y < V; ++y) {
         if (y == a) continue;
+        if (Q1xa[y] > 0.0) nS1 += Qxa[y] + p[y];
+        if (Q1ax[y] > 0.0) nS2 += Qax[y] + (p1[y] > 0.0 ? p[y] + Qxa[y] : 0.0);
         ns_add(&s1, Q1xa[y]);
         ns_add(&s2, Q1ax[y]);
         ns_add(&m1, dmin(p[y], Qxa[y]));       /* pi(x,a,x) */
@@ -275,7 +283,7 @@ void orc_spechub_verify(const double *p, const double *q, int V, int a, int x1, 
         ns_add(&rr, p2[y]);
     }
     double S1 = ns_val(&s1), S2 = ns_val(&s2), R = ns_val(&rr);
-    if (degenerate) S2 = q[a];                 /* all of Q(a, .)'s mass is leftover */
+    if (degenerate) { S2 = q[a]; nS2 = q[a]; } /* all of Q(a, .)'s mass is leftover */
     double hub_after_ax = dmax(p[a] - S2, 0.0);
     out->rate[0] = ns_val(&m1) + dmin(p[a], S2);
     out->rate[1] = ns_val(&m2) + dmin(hub_after_ax, S1);
@@ -283,15 +291,18 @@ void orc_spechub_verify(const double *p, const double *q, int V, int a, int x1, 
 
     int acc = 0;
     if (pair_xa) {
-        acc = accept_test(r1, p[x], Qxa[x], &out->beta[0], &out->margin[0], 1, &out->status);
+        acc = accept_test(r1, p[x], Qxa[x], p[x], Qxa[x], &out->beta[0], &out->cond[0],
+                          &out->margin[0], 1, &out->status);
         if (acc) { out->accept_idx = 0; out->token = x; }
-        int acc2 = accept_test(r2, hub_after_ax, S1, &out->beta[1], &out->margin[1], !acc,
-                               &out->status);
+        int acc2 = accept_test(r2, hub_after_ax, S1, p[a] + nS2, nS1, &out->beta[1], &out->cond[1],
+                               &out->margin[1], !acc, &out->status);
         if (!acc && acc2) { out->accept_idx = 1; out->token = a; acc = 1; }
     } else {
-        acc = accept_test(r1, p1[x], Qax[x], &out->beta[0], &out->margin[0], 1, &out->status);
+        acc = accept_test(r1, p1[x], Qax[x], p[x] + Qxa[x], Qax[x], &out->beta[0], &out->cond[0],
+                          &out->margin[0], 1, &out->status);
         if (acc) { out->accept_idx = 1; out->token = x; }
-        int acc2 = accept_test(r2, p[a], S2, &out->beta[1], &out->margin[1], !acc, &out->status);
+        int acc2 = accept_test(r2, p[a], S2, p[a], nS2, &out->beta[1], &out->cond[1],
+                               &out->margin[1], !acc, &out->status);
         if (!acc && acc2) { out->accept_idx = 0; out->token = a; acc = 1; }
     }
     if (!acc) {
@@ -381,6 +392,8 @@ void orc_rrs_verify(const double *p, const double *q, int V, int x1, int x2, dou
     uint32_t st2 = 0u;
     double A1 = rrs_stage2(p, q, V, x1, without_replacement, p1, q1, &st2);
     nsum m1, m2, w2; ns_init(&m1); ns_init(&m2); ns_init(&w2);
+    double nA1 = 0.0;                           /* term magnitudes of A1, for cond[] only */
+    for (int y = 0; y < V; ++y) if (p[y] > q[y]) nA1 += p[y] + q[y];
     for (int y = 0; y < V; ++y) {
         ns_add(&m1, dmin(p[y], q[y]));
         ns_add(&m2, dmin(p1[y], q1[y]));
@@ -391,12 +404,16 @@ void orc_rrs_verify(const double *p, const double *q, int V, int x1, int x2, dou
     out->rate[1] = A1 * ns_val(&m2);
     out->rate[2] = A1 * ns_val(&w2);
 
-    int acc = accept_test(r1, p[x1], q[x1], &out->beta[0], &out->margin[0], 1, &out->status);
+    int acc = accept_test(r1, p[x1], q[x1], p[x1], q[x1], &out->beta[0], &out->cond[0],
+                          &out->margin[0], 1, &out->status);
     if (acc) { out->accept_idx = 0; out->token = x1; }
     if (!acc) out->status |= st2;
     int acc2 = 0;
     if (A1 > 0.0) {
-        acc2 = accept_test(r2, p1[x2], q1[x2], &out->beta[1], &out->margin[1], !acc, &out->status);
+        /* p_1(x2) = max(p - q, 0)(x2) / A1: both its own subtraction and A1's terms enter */
+        double nN = (p[x2] + q[x2]) / A1 + p1[x2] * nA1 / A1;
+        acc2 = accept_test(r2, p1[x2], q1[x2], nN, q1[x2], &out->beta[1], &out->cond[1],
+                           &out->margin[1], !acc, &out->status);
     } else {
         out->beta[1] = 0.0;
     }

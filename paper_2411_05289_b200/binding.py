@@ -1,0 +1,300 @@
+"""ctypes binding of ``libspechub.so``: argument marshalling only.
+
+Function names and argument meaning follow ``include/spechub.h``.  Tensors are
+torch CUDA tensors; outputs are allocated here with torch (device memory is the
+only thing torch is used for) and returned in small dicts.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+ABI_VERSION = 1
+F32, BF16 = 0, 1
+
+STATUS_BITS = {
+    "NONFINITE": 1,
+    "TOKEN_RANGE": 2,
+    "DEGENERATE_Q": 4,
+    "ZERO_MASS_DRAFT": 8,
+    "ZERO_RESIDUAL": 16,
+}
+
+
+class SpecHubError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("spechub error %d: %s" % (code, msg))
+        self.code = code
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("version", ctypes.c_uint32),
+        ("batch", ctypes.c_int32),
+        ("nodes", ctypes.c_int32),
+        ("vocab", ctypes.c_int32),
+        ("k", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("levels", ctypes.c_int32),
+        ("stride_seq", ctypes.c_int64),
+        ("stride_node", ctypes.c_int64),
+        ("temperature", ctypes.c_float),
+        ("temperature_per_seq", ctypes.c_void_p),
+        ("child", ctypes.c_void_p),
+        ("node_kind", ctypes.c_void_p),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+class _NodeOut(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("accept_idx", "token", "hub", "beta", "rate", "status")]
+
+
+class _SeqOut(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load_library(build_if_missing: bool = True):
+    """Load ``libspechub.so`` (building it with nvcc when it is missing or stale).
+
+    Raises if the library cannot be produced: there is no other implementation to fall back to.
+    """
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if build_if_missing and _build.is_stale():
+        path = _build.build_library()
+    if not os.path.exists(path):
+        raise SpecHubError(-100, "CUDA library %s is missing; run paper_2411_05289_b200.build" % path)
+    lib = ctypes.CDLL(path)
+    vp, i32 = ctypes.c_void_p, ctypes.c_int
+    lib.spechub_draft_sample.restype = i32
+    lib.spechub_draft_sample.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, vp, vp, vp]
+    lib.rrs_draft_sample.restype = i32
+    lib.rrs_draft_sample.argtypes = [ctypes.POINTER(_Desc), vp, vp, i32, vp, vp, vp]
+    lib.spechub_verify_tree.restype = i32
+    lib.spechub_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp,
+                                        ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                        ctypes.c_size_t, vp]
+    lib.rrs_verify_tree.restype = i32
+    lib.rrs_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, i32,
+                                    ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                    ctypes.c_size_t, vp]
+    lib.spechub_workspace_bytes.restype = ctypes.c_size_t
+    lib.spechub_workspace_bytes.argtypes = [ctypes.POINTER(_Desc)]
+    lib.spechub_status_string.restype = ctypes.c_char_p
+    lib.spechub_status_string.argtypes = [i32]
+    lib.spechub_abi_version.restype = i32
+    lib.spechub_abi_version.argtypes = []
+    if lib.spechub_abi_version() != ABI_VERSION:
+        raise SpecHubError(-101, "library ABI %d != binding ABI %d" % (lib.spechub_abi_version(), ABI_VERSION))
+    _lib = lib
+    return lib
+
+
+def abi_version() -> int:
+    return int(load_library().spechub_abi_version())
+
+
+def status_string(code: int) -> str:
+    return load_library().spechub_status_string(int(code)).decode()
+
+
+def _check(code: int):
+    if code != 0:
+        raise SpecHubError(code, status_string(code))
+
+
+@dataclass
+class Tree:
+    """Token tree in level order.  ``child``/``node_kind`` are device tensors or None
+    (None = complete binary tree in heap order, every node verifies)."""
+
+    levels: int
+    child: Optional[torch.Tensor] = None      # int32 [nodes][2]
+    node_kind: Optional[torch.Tensor] = None  # uint8 [nodes]
+
+    @staticmethod
+    def heap(nodes: int, leaves_sample: bool = False, device="cuda") -> "Tree":
+        """Complete binary tree of 2^d - 1 nodes.  With ``leaves_sample`` the last level holds
+        leaves that only draw the bonus token from p (Figure 2 of the paper)."""
+        d = (nodes + 1).bit_length() - 1
+        if (1 << d) - 1 != nodes:
+            raise ValueError("heap trees have 2^d - 1 nodes")
+        kind = None
+        if leaves_sample:
+            kind = torch.zeros(nodes, dtype=torch.uint8)
+            kind[nodes // 2:] = 1
+            kind = kind.to(device)
+        return Tree(levels=d, child=None, node_kind=kind)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _desc(logits: torch.Tensor, tree: Tree, temperature) -> tuple:
+    if logits.dim() != 3 or logits.stride(2) != 1:
+        raise ValueError("logits must be [batch][nodes][vocab] with a contiguous vocabulary axis")
+    if not logits.is_cuda:
+        raise ValueError("logits must live on a CUDA device")
+    if logits.dtype == torch.float32:
+        dt = F32
+    elif logits.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise ValueError("logits must be float32 or bfloat16")
+    B, N, V = logits.shape
+    d = _Desc()
+    d.struct_size = ctypes.sizeof(_Desc)
+    d.version = ABI_VERSION
+    d.batch, d.nodes, d.vocab, d.k = B, N, V, 2
+    d.dtype = dt
+    d.levels = tree.levels
+    d.stride_seq = logits.stride(0) if B > 1 else max(logits.stride(0), (N - 1) * logits.stride(1) + V)
+    d.stride_node = logits.stride(1) if N > 1 else max(logits.stride(1), V)
+    keep = []
+    if isinstance(temperature, torch.Tensor):
+        t = temperature.to(device=logits.device, dtype=torch.float32).contiguous()
+        if t.shape != (B,):
+            raise ValueError("temperature tensor must be [batch]")
+        keep.append(t)
+        d.temperature = 1.0
+        d.temperature_per_seq = t.data_ptr()
+    else:
+        d.temperature = float(temperature)
+        d.temperature_per_seq = None
+    if tree.child is not None:
+        if tree.child.dtype != torch.int32 or tuple(tree.child.shape) != (N, 2) or not tree.child.is_contiguous():
+            raise ValueError("child must be a contiguous int32 [nodes][2] tensor")
+        d.child = tree.child.data_ptr()
+    if tree.node_kind is not None:
+        if tree.node_kind.dtype != torch.uint8 or tuple(tree.node_kind.shape) != (N,):
+            raise ValueError("node_kind must be a uint8 [nodes] tensor")
+        d.node_kind = tree.node_kind.data_ptr()
+    d.flags = 0
+    return d, keep
+
+
+def _same_layout(a: torch.Tensor, b: torch.Tensor):
+    if a.shape != b.shape or a.dtype != b.dtype or a.stride() != b.stride() or a.device != b.device:
+        raise ValueError("target and draft logits must share shape, dtype, strides and device")
+
+
+def _check_uniforms(u, B, N, dev):
+    if u.dtype != torch.float32 or tuple(u.shape) != (B, N, 5) or not u.is_contiguous() or u.device != dev:
+        raise ValueError("uniforms must be a contiguous float32 [batch][nodes][5] tensor on the logits' device")
+
+
+def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
+    """Draw the k = 2 SpecHub drafts of every node.  Returns dict(tokens, hub, prob, status)."""
+    lib = load_library()
+    d, keep = _desc(draft_logits, tree, temperature)
+    B, N, _ = draft_logits.shape
+    dev = draft_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    tokens = torch.empty((B, N, 2), dtype=torch.int32, device=dev)
+    hub = torch.empty((B, N), dtype=torch.int32, device=dev)
+    prob = torch.empty((B, N, 2), dtype=torch.float32, device=dev)
+    status = torch.empty((B, N), dtype=torch.int32, device=dev)
+    _check(lib.spechub_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), _ptr(tokens),
+                                    _ptr(hub), _ptr(prob), _ptr(status), _stream_ptr(stream)))
+    return dict(tokens=tokens, hub=hub, prob=prob, status=status)
+
+
+def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bool, temperature=1.0,
+                     stream=None):
+    """Draw the k = 2 RRS / RRSw drafts of every node.  Returns dict(tokens, status)."""
+    lib = load_library()
+    d, keep = _desc(draft_logits, tree, temperature)
+    B, N, _ = draft_logits.shape
+    dev = draft_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    tokens = torch.empty((B, N, 2), dtype=torch.int32, device=dev)
+    status = torch.empty((B, N), dtype=torch.int32, device=dev)
+    _check(lib.rrs_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
+                                int(bool(without_replacement)), _ptr(tokens), _ptr(status),
+                                _stream_ptr(stream)))
+    return dict(tokens=tokens, status=status)
+
+
+def alloc_verify_outputs(B, N, levels, dev):
+    """Device buffers for one verify call (reusable across calls of the same shape)."""
+    return dict(
+        accept_idx=torch.empty((B, N), dtype=torch.int32, device=dev),
+        token=torch.empty((B, N), dtype=torch.int32, device=dev),
+        hub=torch.empty((B, N), dtype=torch.int32, device=dev),
+        beta=torch.empty((B, N, 2), dtype=torch.float32, device=dev),
+        rate=torch.empty((B, N, 3), dtype=torch.float32, device=dev),
+        status=torch.empty((B, N), dtype=torch.int32, device=dev),
+        n_accepted=torch.empty((B,), dtype=torch.int32, device=dev),
+        n_emitted=torch.empty((B,), dtype=torch.int32, device=dev),
+        path_nodes=torch.empty((B, levels), dtype=torch.int32, device=dev),
+        path_tokens=torch.empty((B, levels), dtype=torch.int32, device=dev),
+    )
+
+
+def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream,
+            out):
+    lib = load_library()
+    _same_layout(target_logits, draft_logits)
+    d, keep = _desc(target_logits, tree, temperature)
+    B, N, _ = target_logits.shape
+    dev = target_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    if (draft_tokens.dtype != torch.int32 or tuple(draft_tokens.shape) != (B, N, 2)
+            or not draft_tokens.is_contiguous() or draft_tokens.device != dev):
+        raise ValueError("draft_tokens must be a contiguous int32 [batch][nodes][2] tensor")
+    if out is None:
+        out = alloc_verify_outputs(B, N, tree.levels, dev)
+    no = _NodeOut(*[out[k].data_ptr() for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
+    so = _SeqOut(*[out[k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])
+    ws_bytes = lib.spechub_workspace_bytes(ctypes.byref(d))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
+    common = (ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms))
+    tail = (ctypes.byref(no), ctypes.byref(so), _ptr(ws), ws_bytes, _stream_ptr(stream))
+    if method == "spechub":
+        _check(lib.spechub_verify_tree(*common, *tail))
+    else:
+        _check(lib.rrs_verify_tree(*common, 1 if method == "rrsw" else 0, *tail))
+    return out
+
+
+def spechub_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
+                        temperature=1.0, stream=None, out=None):
+    """SpecHub verification of every node and the tree walk.  Returns the dict of output
+    tensors (see ``alloc_verify_outputs``); pass ``out`` to reuse buffers."""
+    return _verify("spechub", target_logits, draft_logits, draft_tokens, uniforms, tree, temperature,
+                   stream, out)
+
+
+def rrs_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
+                    without_replacement: bool, temperature=1.0, stream=None, out=None):
+    """RRS / RRSw verification of every node and the tree walk."""
+    return _verify("rrsw" if without_replacement else "rrs", target_logits, draft_logits, draft_tokens,
+                   uniforms, tree, temperature, stream, out)
+
+
+def workspace_bytes(logits, tree: Tree, temperature=1.0) -> int:
+    d, _ = _desc(logits, tree, temperature)
+    return int(load_library().spechub_workspace_bytes(ctypes.byref(d)))

@@ -1,0 +1,215 @@
+// C ABI of the library (see include/spechub.h): host-side argument checks and
+// kernel launches.  Nothing here allocates or synchronises.
+#include <cuda_runtime.h>
+#include <math.h>
+
+#include "spechub.h"
+#include "spechub_common.cuh"
+#include "spechub_stream.cuh"
+
+namespace {
+
+using namespace spechub;
+
+int check_desc(const spechub_desc *d) {
+    if (!d) return SPECHUB_ERR_NULL;
+    if (d->struct_size != sizeof(spechub_desc) || d->version != SPECHUB_ABI_VERSION)
+        return SPECHUB_ERR_VERSION;
+    if (d->batch < 0 || d->nodes < 1 || d->vocab < 2 || d->k != 2 || d->levels < 1)
+        return SPECHUB_ERR_SHAPE;
+    if (d->dtype != SPECHUB_F32 && d->dtype != SPECHUB_BF16) return SPECHUB_ERR_DTYPE;
+    if (d->stride_node < d->vocab) return SPECHUB_ERR_STRIDE;
+    if (d->nodes > 1 && d->stride_seq < d->stride_node * (int64_t)(d->nodes - 1) + d->vocab)
+        return SPECHUB_ERR_STRIDE;
+    if (d->nodes == 1 && d->batch > 1 && d->stride_seq < d->vocab) return SPECHUB_ERR_STRIDE;
+    if (!d->temperature_per_seq && !(d->temperature > 0.f && isfinite(d->temperature)))
+        return SPECHUB_ERR_TEMPERATURE;
+    if (d->flags != 0) return SPECHUB_ERR_SHAPE;
+    if ((int64_t)d->batch * d->nodes > 0x7fffffffLL) return SPECHUB_ERR_SHAPE;
+    return SPECHUB_OK;
+}
+
+// rows whose every start is 16-byte aligned take the 128-bit load path
+bool rows_aligned(const spechub_desc *d, const void *base) {
+    const int esz = d->dtype == SPECHUB_BF16 ? 2 : 4;
+    const int per16 = 16 / esz;
+    return (reinterpret_cast<uintptr_t>(base) % 16 == 0) && (d->stride_node % per16 == 0) &&
+           (d->stride_seq % per16 == 0);
+}
+
+int threads_for(const spechub_desc *d) {
+    const int vw = d->dtype == SPECHUB_BF16 ? 8 : 4;
+    const int nvec = (d->vocab + vw - 1) / vw;
+    if (nvec >= 8192) return 512;
+    if (nvec >= 2048) return 256;
+    if (nvec >= 128) return 128;
+    if (nvec >= 64) return 64;
+    return 32;
+}
+
+RowArgs base_args(const spechub_desc *d) {
+    RowArgs a = {};
+    a.temperature_per_seq = d->temperature_per_seq;
+    a.node_kind = d->node_kind;
+    a.temperature = d->temperature;
+    a.nodes = d->nodes;
+    a.vocab = d->vocab;
+    a.stride_seq = d->stride_seq;
+    a.stride_node = d->stride_node;
+    return a;
+}
+
+int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH; }
+
+int draft_common(const spechub_desc *d, const void *draft_logits, const float *uniforms, int method,
+                 int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
+                 void *stream) {
+    const int rc = check_desc(d);
+    if (rc != SPECHUB_OK) return rc;
+    if (d->batch == 0) return SPECHUB_OK;  // nothing to do; pointers are not looked at
+    if (!draft_logits || !uniforms || !draft_tokens) return SPECHUB_ERR_NULL;
+    RowArgs a = base_args(d);
+    a.draft = draft_logits;
+    a.uniforms = uniforms;
+    a.draft_tokens_out = draft_tokens;
+    a.hub = hub;
+    a.draft_prob = draft_prob;
+    a.status = status;
+    const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
+    const int th = threads_for(d);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool al = rows_aligned(d, draft_logits);
+    if (d->dtype == SPECHUB_BF16) {
+        if (al) draft_rows_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(a, method);
+        else draft_rows_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(a, method);
+    } else {
+        if (al) draft_rows_kernel<float, true><<<rows, th, 0, s>>>(a, method);
+        else draft_rows_kernel<float, false><<<rows, th, 0, s>>>(a, method);
+    }
+    return launch_status();
+}
+
+template <int METHOD>
+void launch_verify(const spechub_desc *d, const RowArgs &a, bool al, unsigned rows, int th,
+                   cudaStream_t s) {
+    if (d->dtype == SPECHUB_BF16) {
+        if (al) verify_rows_kernel<__nv_bfloat16, true, METHOD><<<rows, th, 0, s>>>(a);
+        else verify_rows_kernel<__nv_bfloat16, false, METHOD><<<rows, th, 0, s>>>(a);
+    } else {
+        if (al) verify_rows_kernel<float, true, METHOD><<<rows, th, 0, s>>>(a);
+        else verify_rows_kernel<float, false, METHOD><<<rows, th, 0, s>>>(a);
+    }
+}
+
+int verify_common(const spechub_desc *d, const void *target_logits, const void *draft_logits,
+                  const int32_t *draft_tokens, const float *uniforms, int method,
+                  const spechub_node_out *no, const spechub_seq_out *so, void *workspace,
+                  size_t workspace_bytes, void *stream) {
+    const int rc = check_desc(d);
+    if (rc != SPECHUB_OK) return rc;
+    if (d->batch == 0) return SPECHUB_OK;  // nothing to do; pointers are not looked at
+    if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !no || !no->accept_idx ||
+        !no->token)
+        return SPECHUB_ERR_NULL;
+    if (workspace_bytes < spechub_workspace_bytes(d)) return SPECHUB_ERR_WORKSPACE;
+    (void)workspace;
+    RowArgs a = base_args(d);
+    a.target = target_logits;
+    a.draft = draft_logits;
+    a.uniforms = uniforms;
+    a.draft_tokens_in = draft_tokens;
+    a.hub = no->hub;
+    a.accept_idx = no->accept_idx;
+    a.token = no->token;
+    a.beta = no->beta;
+    a.rate = no->rate;
+    a.status = no->status;
+    const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
+    const int th = threads_for(d);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool al = rows_aligned(d, target_logits) && rows_aligned(d, draft_logits);
+    if (method == kSpecHub) launch_verify<kSpecHub>(d, a, al, rows, th, s);
+    else if (method == kRRS) launch_verify<kRRS>(d, a, al, rows, th, s);
+    else launch_verify<kRRSw>(d, a, al, rows, th, s);
+    int lrc = launch_status();
+    if (lrc != SPECHUB_OK) return lrc;
+    if (so && (so->n_accepted || so->n_emitted || so->path_nodes || so->path_tokens)) {
+        WalkArgs w;
+        w.accept_idx = no->accept_idx;
+        w.token = no->token;
+        w.child = d->child;
+        w.node_kind = d->node_kind;
+        w.n_accepted = so->n_accepted;
+        w.n_emitted = so->n_emitted;
+        w.path_nodes = so->path_nodes;
+        w.path_tokens = so->path_tokens;
+        w.batch = d->batch;
+        w.nodes = d->nodes;
+        w.levels = d->levels;
+        walk_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(w);
+        lrc = launch_status();
+    }
+    return lrc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int spechub_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                         int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
+                         void *stream) {
+    return draft_common(desc, draft_logits, uniforms, kSpecHub, draft_tokens, hub, draft_prob, status,
+                        stream);
+}
+
+int rrs_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                     int without_replacement, int32_t *draft_tokens, uint32_t *status, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    return draft_common(desc, draft_logits, uniforms, without_replacement ? kRRSw : kRRS,
+                        draft_tokens, nullptr, nullptr, status, stream);
+}
+
+int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
+                        const void *draft_logits, const int32_t *draft_tokens,
+                        const float *uniforms, const spechub_node_out *node_out,
+                        const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                        void *stream) {
+    return verify_common(desc, target_logits, draft_logits, draft_tokens, uniforms, kSpecHub,
+                         node_out, seq_out, workspace, workspace_bytes, stream);
+}
+
+int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                    const int32_t *draft_tokens, const float *uniforms, int without_replacement,
+                    const spechub_node_out *node_out, const spechub_seq_out *seq_out,
+                    void *workspace, size_t workspace_bytes, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    return verify_common(desc, target_logits, draft_logits, draft_tokens, uniforms,
+                         without_replacement ? kRRSw : kRRS, node_out, seq_out, workspace,
+                         workspace_bytes, stream);
+}
+
+size_t spechub_workspace_bytes(const spechub_desc *desc) {
+    (void)desc;
+    return 0;
+}
+
+const char *spechub_status_string(int code) {
+    switch (code) {
+        case SPECHUB_OK: return "ok";
+        case SPECHUB_ERR_NULL: return "a required pointer is NULL";
+        case SPECHUB_ERR_VERSION: return "descriptor struct_size/version mismatch";
+        case SPECHUB_ERR_SHAPE: return "bad shape: need batch >= 0, nodes >= 1, vocab >= 2, k == 2, levels >= 1, flags == 0";
+        case SPECHUB_ERR_DTYPE: return "dtype must be SPECHUB_F32 or SPECHUB_BF16";
+        case SPECHUB_ERR_STRIDE: return "strides too small for the given shape";
+        case SPECHUB_ERR_TEMPERATURE: return "temperature must be finite and > 0";
+        case SPECHUB_ERR_WORKSPACE: return "workspace smaller than spechub_workspace_bytes()";
+        case SPECHUB_ERR_LAUNCH: return "kernel launch failed";
+        case SPECHUB_ERR_METHOD: return "without_replacement must be 0 or 1";
+        default: return "unknown status";
+    }
+}
+
+int spechub_abi_version(void) { return SPECHUB_ABI_VERSION; }
+
+}  // extern "C"

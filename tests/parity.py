@@ -1,0 +1,228 @@
+"""GPU-vs-oracle comparison rules shared by the parity tests, the smoke check and nothing else.
+
+The rule: decisions (accept / reject), hub and token ids must be identical,
+except where a uniform lies within NEAR = 1e-6 of the threshold it is compared
+with -- then the GPU may sit on the other side of that one threshold, and what
+follows is checked against the oracle re-run on that side.  For a sampled token
+"threshold" means an edge of the token's interval in the oracle's fp64 CDF.
+
+Probabilities: |gpu - oracle| <= RTOL * |oracle| + ATOL with RTOL = 1e-5.  The
+absolute term covers values that the fp32 path forms as a difference of O(1)
+sums (rates, the hub's leftover mass): each sum carries a relative error of a
+few fp32 ulps times log2(V) from the fixed-order tree summation, i.e. about
+1e-6 absolute on quantities bounded by 1.
+
+Conditioning.  An acceptance probability N/D whose numerator is a difference
+(p(x) - q(x), p(a) - S2) is ill-conditioned when the operands nearly cancel:
+a relative error EPS in every fp32 p(y), q(y) moves N/D by EPS * cond, where
+cond = (|N| + beta |D|) / D is reported by the oracle (|.| = sum of the
+magnitudes of the terms).  EPS = 1e-6 is the fp32 path's bound on a single
+probability: 2 ulp from ex2.approx, up to 2^-20 absolute on an exponent of
+magnitude <= 20 from the FMA that forms it, and the rounding of 1/Z.  So the
+tolerance of beta_i is RTOL * beta_i + EPS * cond_i, and the band around the
+threshold inside which the GPU may decide the other way is
+max(NEAR, EPS * cond_i): 1e-6 for a well-conditioned test, wider only where
+fp32 cannot resolve the threshold itself.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+
+NEAR = 1e-6
+RTOL = 1e-5
+ATOL = 1e-6
+EPS = 1e-6
+
+FATAL = oracle.STATUS_BITS["NONFINITE"] | oracle.STATUS_BITS["TOKEN_RANGE"]
+
+
+class Stats:
+    def __init__(self):
+        self.rows = 0
+        self.exact = 0
+        self.exempt_test = 0
+        self.exempt_token = 0
+        self.wide_band = 0
+        self.max_rel = 0.0
+
+    def __repr__(self):
+        return "rows=%d exact=%d exempt_test=%d exempt_token=%d wide_band=%d max_prob_err=%.2e" % (
+            self.rows, self.exact, self.exempt_test, self.exempt_token, self.wide_band, self.max_rel)
+
+
+def _close(g, o, what, ctx, stats, atol=ATOL):
+    g = np.asarray(g, np.float64)
+    o = np.asarray(o, np.float64)
+    err = np.abs(g - o)
+    tol = RTOL * np.abs(o) + atol
+    if not np.all(err <= tol):
+        raise AssertionError("%s mismatch %s: gpu=%s oracle=%s" % (what, ctx, g, o))
+    stats.max_rel = max(stats.max_rel, float(np.max(err / (np.abs(o) + atol))))
+
+
+def _token_consistent(w, tok, u):
+    """Is `tok` an admissible inverse-CDF draw of weights w with uniform u, within NEAR?"""
+    if tok < 0 or tok >= len(w):
+        return False
+    lo, hi = oracle.cdf_interval(w, tok)
+    return lo - NEAR <= u <= hi + NEAR
+
+
+def check_draft_row(method, lq_row, T, u, g_tokens, g_hub, g_prob, g_status, o_tokens, o_hub, o_prob,
+                    o_status, ctx, stats):
+    """One row of the draft step.  o_* come from oracle.draft_batch on the same inputs."""
+    stats.rows += 1
+    if o_status & FATAL:
+        assert g_status & FATAL and tuple(g_tokens) == (-1, -1), ("draft fatal row", ctx, g_tokens, g_status)
+        return
+    assert not (g_status & FATAL), ("unexpected fatal status", ctx, g_status)
+    if method == "spechub":
+        assert g_hub == o_hub, ("hub", ctx, g_hub, o_hub)
+    if tuple(g_tokens) == tuple(o_tokens):
+        stats.exact += 1
+        assert g_status == o_status, ("status", ctx, g_status, o_status)
+        if method == "spechub" and g_prob is not None:
+            _close(g_prob, o_prob, "draft_prob", ctx, stats, atol=1e-9)
+        return
+    # tokens differ: the GPU's choices must each be admissible given its earlier choices
+    q, st = oracle.softmax(lq_row, T)
+    stats.exempt_token += 1
+    x1, x2 = int(g_tokens[0]), int(g_tokens[1])
+    assert _token_consistent(q, x1, u[0]), ("x1 not admissible", ctx, g_tokens, o_tokens)
+    if method == "spechub":
+        a = o_hub
+        if x1 != a:
+            assert x2 == a, ("x2 must be the hub", ctx, g_tokens)
+        else:
+            w = q.copy(); w[a] = 0.0
+            assert _token_consistent(w, x2, u[1]), ("x2 not admissible", ctx, g_tokens, o_tokens)
+    elif method == "rrs":
+        assert _token_consistent(q, x2, u[1]), ("x2 not admissible", ctx, g_tokens, o_tokens)
+    else:
+        w = q.copy(); w[x1] = 0.0
+        assert _token_consistent(w, x2, u[1]), ("x2 not admissible", ctx, g_tokens, o_tokens)
+
+
+def _oracle_row(method, p, q, a, x1, x2, r1, r2, ur):
+    if method == "spechub":
+        return oracle.spechub_verify(p, q, a, x1, x2, r1, r2, ur)
+    return oracle.rrs_verify(p, q, x1, x2, r1, r2, ur, method == "rrsw")
+
+
+def check_verify_row(method, lp_row, lq_row, T, tokens, u, leaf, g, o, ctx, stats):
+    """One row of verification.  g: dict of python scalars/arrays from the GPU
+    (accept_idx, token, hub, beta[2], rate[3], status); o: the oracle's NODE_DTYPE record."""
+    stats.rows += 1
+    o_st = int(o["status"])
+    if o_st & FATAL:
+        assert g["status"] & FATAL == o_st & FATAL, ("fatal status", ctx, g["status"], o_st)
+        assert g["token"] == -1 and g["accept_idx"] == -1, ("fatal row output", ctx, g)
+        return
+    assert not (g["status"] & FATAL), ("unexpected fatal status", ctx, g["status"])
+    r1, r2, ur = float(u[2]), float(u[3]), float(u[4])
+    if leaf:
+        assert g["accept_idx"] == -1
+        if g["token"] == o["token"]:
+            stats.exact += 1
+            return
+        p, _ = oracle.softmax(lp_row, T)
+        assert _token_consistent(p, g["token"], ur), ("leaf token", ctx, g["token"], o["token"])
+        stats.exempt_token += 1
+        return
+    if method == "spechub":
+        assert g["hub"] == o["hub"], ("hub", ctx, g["hub"], o["hub"])
+    # probabilities first: they do not depend on the uniforms
+    for i in range(2):
+        _close(g["beta"][i], o["beta"][i], "beta[%d]" % i, ctx, stats, atol=ATOL + EPS * float(o["cond"][i]))
+    _close(g["rate"], o["rate"], "rate", ctx, stats)
+    if g["accept_idx"] == o["accept_idx"] and g["token"] == o["token"]:
+        stats.exact += 1
+        soft = oracle.STATUS_BITS["ZERO_RESIDUAL"]
+        assert (g["status"] | soft) == (o_st | soft), ("status", ctx, g["status"], o_st)
+        return
+    # something differs: find the admissible alternative
+    p, _ = oracle.softmax(lp_row, T)
+    q, _ = oracle.softmax(lq_row, T)
+    a = int(o["hub"])
+    x1, x2 = int(tokens[0]), int(tokens[1])
+    cands = [(r1, r2)]
+    m1 = float(o["margin"][0])
+    band1 = max(NEAR, EPS * float(o["cond"][0]))
+    r1s = [r1] + ([min(max(r1 - 2 * m1 - 1e-9, 0.0), 1.0), min(r1 + 2 * m1 + 1e-9, 1.0)] if m1 <= band1 else [])
+    for rr1 in r1s:
+        o1 = _oracle_row(method, p, q, a, x1, x2, rr1, r2, ur)
+        mm2 = float(o1["margin"][1])
+        band2 = max(NEAR, EPS * float(o1["cond"][1]))
+        if band1 > NEAR or band2 > NEAR:
+            stats.wide_band += 1
+        r2s = [r2] + ([min(max(r2 - 2 * mm2 - 1e-9, 0.0), 1.0), min(r2 + 2 * mm2 + 1e-9, 1.0)] if mm2 <= band2 else [])
+        for rr2 in r2s:
+            cands.append((rr1, rr2))
+    for (rr1, rr2) in cands:
+        alt = _oracle_row(method, p, q, a, x1, x2, rr1, rr2, ur)
+        if alt["accept_idx"] != g["accept_idx"]:
+            continue
+        if g["accept_idx"] >= 0:
+            if alt["token"] == g["token"]:
+                stats.exempt_test += 1
+                return
+            continue
+        # both rejected: the residual token must be admissible
+        if alt["token"] == g["token"]:
+            stats.exempt_test += 1
+            return
+        if alt["status"] & oracle.STATUS_BITS["ZERO_RESIDUAL"]:
+            w = p
+        elif method == "spechub":
+            w = oracle.spechub_residual(p, q, a)
+        else:
+            w = oracle.rrs_residual(p, q, x1, method == "rrsw")
+        if _token_consistent(w, g["token"], ur):
+            stats.exempt_token += 1
+            return
+    raise AssertionError("decision/token mismatch %s: gpu=(%d,%d) oracle=(%d,%d) margins=%s u=%s" % (
+        ctx, g["accept_idx"], g["token"], o["accept_idx"], o["token"], o["margin"], (r1, r2, ur)))
+
+
+def temps_array(T, B):
+    t = np.asarray(T, np.float32)
+    return np.full(B, float(t), np.float32) if t.ndim == 0 else t
+
+
+def check_verify(method, lp, lq, T, tokens, uniforms, node_kind, gpu, stats=None, label=""):
+    """All rows of a [B][N][V] problem.  gpu: dict of numpy arrays as returned by the binding."""
+    stats = stats or Stats()
+    B, N, V = lp.shape
+    t = temps_array(T, B)
+    o = oracle.verify_batch(method, lp, lq, t, tokens, uniforms, node_kind)
+    for b in range(B):
+        for n in range(N):
+            g = dict(accept_idx=int(gpu["accept_idx"][b, n]), token=int(gpu["token"][b, n]),
+                     hub=int(gpu["hub"][b, n]), beta=gpu["beta"][b, n], rate=gpu["rate"][b, n],
+                     status=int(gpu["status"][b, n]))
+            leaf = node_kind is not None and node_kind[n] == 1
+            check_verify_row(method, lp[b, n], lq[b, n], float(t[b]), tokens[b, n], uniforms[b, n], leaf,
+                             g, o[b, n], "%s[%s b=%d n=%d V=%d]" % (label, method, b, n, V), stats)
+    return stats, o
+
+
+def check_draft(method, lq, T, uniforms, gpu, stats=None, label=""):
+    stats = stats or Stats()
+    B, N, V = lq.shape
+    t = temps_array(T, B)
+    o = oracle.draft_batch(method, lq, t, uniforms)
+    for b in range(B):
+        for n in range(N):
+            gp = gpu["prob"][b, n] if "prob" in gpu and gpu["prob"] is not None else None
+            gh = int(gpu["hub"][b, n]) if "hub" in gpu and gpu["hub"] is not None else -1
+            check_draft_row(method, lq[b, n], float(t[b]), uniforms[b, n], gpu["tokens"][b, n], gh, gp,
+                            int(gpu["status"][b, n]), o["tokens"][b, n], int(o["hub"][b, n]),
+                            o["prob"][b, n], int(o["status"][b, n]),
+                            "%s[%s b=%d n=%d V=%d]" % (label, method, b, n, V), stats)
+    return stats, o
+
+
+def to_numpy(d):
+    return {k: (v.detach().cpu().numpy() if hasattr(v, "detach") else v) for k, v in d.items()}

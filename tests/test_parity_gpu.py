@@ -1,0 +1,328 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle.
+
+Small problems are compared row by row on every output; the five benchmark
+configurations run on the GPU at full size, in the launch configuration the
+benchmark times, and are compared on sampled rows.
+"""
+import os
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+import oracle  # noqa: E402
+import workloads  # noqa: E402
+import parity  # noqa: E402
+
+METHODS = ("spechub", "rrs", "rrsw")
+
+
+@pytest.fixture(scope="module")
+def sh():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2411_05289_b200 as lib
+
+    lib.load_library()
+    return lib
+
+
+def gpu_draft(sh, method, tq, un, tree, T):
+    if method == "spechub":
+        return sh.spechub_draft_sample(tq, un, tree, T)
+    return sh.rrs_draft_sample(tq, un, tree, method == "rrsw", T)
+
+
+def gpu_verify(sh, method, tp, tq, tok, un, tree, T, out=None):
+    if method == "spechub":
+        return sh.spechub_verify_tree(tp, tq, tok, un, tree, T, out=out)
+    return sh.rrs_verify_tree(tp, tq, tok, un, tree, method == "rrsw", T, out=out)
+
+
+def padded(x, dtype, pad_to, device="cuda"):
+    """Device copy of host fp32 [B][N][V] in the storage dtype; rows padded to a multiple of
+    `pad_to` elements (0 = dense rows, which are unaligned when V is odd)."""
+    B, N, V = x.shape
+    t = workloads.to_device(x, dtype, device)
+    if not pad_to:
+        return t
+    Vp = (V + pad_to - 1) // pad_to * pad_to
+    buf = torch.full((B, N, Vp), float("nan"), dtype=t.dtype, device=device)
+    buf[:, :, :V] = t
+    return buf[:, :, :V]
+
+
+def run_case(sh, lp, lq, dtype, T, un, paper_layout, pad_to=0, methods=METHODS, label=""):
+    B, N, V = lp.shape
+    Tt = torch.tensor(np.asarray(T, np.float32), device="cuda") if np.ndim(T) else float(T)
+    tp, tq = padded(lp, dtype, pad_to), padded(lq, dtype, pad_to)
+    und = torch.from_numpy(un).cuda()
+    kind = workloads.paper_node_kind(N) if paper_layout else None
+    tree = sh.Tree.heap(N, leaves_sample=paper_layout)
+    total = parity.Stats()
+    for m in methods:
+        d = parity.to_numpy(gpu_draft(sh, m, tq, und, tree, Tt))
+        st, od = parity.check_draft(m, lq, T, un, d, label=label)
+        # verification parity is checked on the oracle's drafts so that both sides see the same pair
+        tok = od["tokens"].copy()
+        out = parity.to_numpy(gpu_verify(sh, m, tp, tq, torch.from_numpy(tok).cuda(), und, tree, Tt))
+        torch.cuda.synchronize()
+        sv, ov = parity.check_verify(m, lp, lq, T, tok, un, kind, out, label=label)
+        w = oracle.walk(out["accept_idx"], out["token"], tree.levels, node_kind=kind)
+        for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+            np.testing.assert_array_equal(out[k], w[k], err_msg="%s walk %s" % (label, k))
+        for s in (st, sv):
+            total.rows += s.rows; total.exact += s.exact
+            total.exempt_test += s.exempt_test; total.exempt_token += s.exempt_token
+            total.max_rel = max(total.max_rel, s.max_rel)
+    return total
+
+
+def random_logits(rng, B, N, V, dtype, sd=2.0, sigma=1.0):
+    lp = rng.normal(0, sd, (B, N, V)).astype(np.float32)
+    lq = lp + rng.normal(0, sigma, (B, N, V)).astype(np.float32)
+    return workloads.round_to_storage(lp, dtype), workloads.round_to_storage(lq, dtype)
+
+
+def random_uniforms(rng, B, N):
+    return (rng.integers(0, 1 << 24, (B, N, 5)).astype(np.float32) * np.float32(2.0 ** -24))
+
+
+# ------------------------------------------------------------------------------------------------
+# small shapes: every tile boundary, ragged tails, unaligned rows, both dtypes, both layouts
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("V", [2, 3, 5, 8, 33, 257, 1000, 1031, 4099, 9000, 20011])
+def test_small_shapes(sh, V, dtype):
+    rng = np.random.default_rng(V * 7 + (dtype == "bf16"))
+    B, N = (3, 7) if V > 1000 else (6, 7)
+    lp, lq = random_logits(rng, B, N, V, dtype)
+    un = random_uniforms(rng, B, N)
+    T = np.array([1.0, 0.6, 1.3, 0.8, 1.0, 2.0][:B], np.float32)
+    s = run_case(sh, lp, lq, dtype, T, un, paper_layout=False, pad_to=0, label="dense-unaligned")
+    s2 = run_case(sh, lp, lq, dtype, 1.0, un, paper_layout=True, pad_to=8, label="paper-aligned")
+    assert s.rows and s2.rows
+
+
+def test_peaked_rows_keep_precision(sh):
+    """q close to one-hot: 1 - q(a) must come from a direct sum, not from 1 - q(a)."""
+    rng = np.random.default_rng(5)
+    B, N, V = 4, 3, 5000
+    lp, lq = random_logits(rng, B, N, V, "fp32")
+    for b in range(B):
+        lq[b, :, 17 + b] += 12.0 + 4 * b
+    un = random_uniforms(rng, B, N)
+    un[:, :, 0] = 0.5  # x1 = hub, so the second draw and c = q(a)/(1-q(a)) are exercised
+    run_case(sh, lp, lq, "fp32", 1.0, un, paper_layout=False, label="peaked")
+
+
+# ------------------------------------------------------------------------------------------------
+# degenerate and malformed rows
+# ------------------------------------------------------------------------------------------------
+
+def test_degenerate_rows(sh):
+    rng = np.random.default_rng(11)
+    V = 2048
+    lp, lq = random_logits(rng, 1, 7, V, "bf16")
+    lq[0, 0] = lp[0, 0]                                   # p = q: never rejects
+    lq[0, 1] = -np.inf; lq[0, 1, 77] = 0.0                # one-hot q
+    lq[0, 2] = -60.0; lq[0, 2, 5] = 0.0                   # nearly one-hot q
+    lp[0, 3, :1024] = -np.inf; lq[0, 3, 1024:] = -np.inf  # disjoint supports
+    lq[0, 4] = workloads.round_to_storage(rng.normal(0, 0.01, V).astype(np.float32), "bf16")
+    lp[0, 5] = np.round(lp[0, 5] * 2) / 2; lq[0, 5] = np.round(lq[0, 5] * 2) / 2  # many exact ties
+    lq[0, 6] = 0.0                                        # exactly uniform q: hub = id 0
+    for seed in range(4):
+        un = random_uniforms(np.random.default_rng(seed), 1, 7)
+        run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=False, label="degenerate")
+
+
+def test_flagged_rows(sh):
+    rng = np.random.default_rng(12)
+    V = 1000
+    lp, lq = random_logits(rng, 1, 7, V, "fp32")
+    lp[0, 0, 3] = np.nan
+    lq[0, 1, 9] = np.inf
+    lq[0, 2] = -np.inf
+    un = random_uniforms(rng, 1, 7)
+    tree = sh.Tree.heap(7)
+    tp, tq, und = workloads.to_device(lp, "fp32"), workloads.to_device(lq, "fp32"), torch.from_numpy(un).cuda()
+    for m in METHODS:
+        d = parity.to_numpy(gpu_draft(sh, m, tq, und, tree, 1.0))
+        st, od = parity.check_draft(m, lq, 1.0, un, d)
+        assert d["status"][0, 1] & 1 and d["status"][0, 2] & 1 and not d["status"][0, 0] & 1
+        tok = od["tokens"].copy()
+        tok[0, 0] = tok[0, 1] = tok[0, 2] = (1, 2)
+        tok[0, 3] = (V, 0)            # out of range
+        tok[0, 4] = (-1, 5)
+        hub4 = int(np.argmax(lq[0, 5]))
+        tok[0, 5] = (hub4, hub4)      # SpecHub: pair holds the hub twice
+        out = parity.to_numpy(gpu_verify(sh, m, tp, tq, torch.from_numpy(tok).cuda(), und, tree, 1.0))
+        parity.check_verify(m, lp, lq, 1.0, tok, un, None, out)
+        assert (out["status"][0, :3] & 1).all()
+        assert (out["status"][0, 3:5] & 2).all()
+        assert (out["token"][0, :5] == -1).all()
+        assert out["n_emitted"][0] == 0
+
+
+def test_argument_errors(sh):
+    import ctypes
+
+    from paper_2411_05289_b200 import binding
+
+    lib = sh.load_library()
+    x = torch.zeros((2, 3, 64), dtype=torch.float32, device="cuda")
+    d, _ = binding._desc(x, sh.Tree.heap(3), 1.0)
+    un = torch.zeros((2, 3, 5), device="cuda")
+    tok = torch.zeros((2, 3, 2), dtype=torch.int32, device="cuda")
+    vp = ctypes.c_void_p
+    call = lambda dd: lib.spechub_draft_sample(ctypes.byref(dd), vp(x.data_ptr()), vp(un.data_ptr()),
+                                               vp(tok.data_ptr()), None, None, None, None)
+    assert call(d) == 0
+    for field, val, code in [("k", 3, -3), ("vocab", 1, -3), ("dtype", 7, -4), ("version", 9, -2),
+                             ("stride_node", 8, -5), ("temperature", 0.0, -6), ("levels", 0, -3),
+                             ("flags", 1, -3)]:
+        dd, _ = binding._desc(x, sh.Tree.heap(3), 1.0)
+        setattr(dd, field, val)
+        assert call(dd) == code, field
+    assert lib.spechub_draft_sample(ctypes.byref(d), None, vp(un.data_ptr()), vp(tok.data_ptr()),
+                                    None, None, None, None) == -1
+    assert lib.rrs_draft_sample(ctypes.byref(d), vp(x.data_ptr()), vp(un.data_ptr()), 2,
+                                vp(tok.data_ptr()), None, None) == -9
+    torch.cuda.synchronize()
+    # empty batch is a no-op
+    e = torch.zeros((0, 3, 64), device="cuda")
+    out = sh.spechub_draft_sample(e, torch.zeros((0, 3, 5), device="cuda"), sh.Tree.heap(3))
+    assert out["tokens"].shape == (0, 3, 2)
+
+
+def test_custom_child_table_and_determinism(sh):
+    rng = np.random.default_rng(21)
+    B, N, V = 16, 5, 3000
+    lp, lq = random_logits(rng, B, N, V, "bf16", sigma=0.3)
+    un = random_uniforms(rng, B, N)
+    child = np.array([[1, 2], [3, -1], [4, -1], [-1, -1], [-1, -1]], np.int32)  # unbalanced tree
+    kind = np.array([0, 0, 0, 1, 0], np.uint8)
+    tree = sh.Tree(levels=3, child=torch.from_numpy(child).cuda(), node_kind=torch.from_numpy(kind).cuda())
+    tp, tq, und = workloads.to_device(lp, "bf16"), workloads.to_device(lq, "bf16"), torch.from_numpy(un).cuda()
+    d = gpu_draft(sh, "spechub", tq, und, tree, 1.0)
+    o1 = parity.to_numpy(gpu_verify(sh, "spechub", tp, tq, d["tokens"], und, tree, 1.0))
+    o2 = parity.to_numpy(gpu_verify(sh, "spechub", tp, tq, d["tokens"], und, tree, 1.0))
+    for k in o1:
+        np.testing.assert_array_equal(o1[k], o2[k], err_msg=k)  # bit-identical across runs
+    w = oracle.walk(o1["accept_idx"], o1["token"], 3, child=child, node_kind=kind)
+    for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+        np.testing.assert_array_equal(o1[k], w[k])
+    parity.check_verify("spechub", lp, lq, 1.0, parity.to_numpy(d)["tokens"], un, kind, o1)
+
+
+# ------------------------------------------------------------------------------------------------
+# the benchmark configurations
+# ------------------------------------------------------------------------------------------------
+
+def test_config1_full(sh):
+    cfg = workloads.CONFIGS["c1"]
+    lp, lq = workloads.host_logits(cfg)
+    un = workloads.host_uniforms(cfg)
+    for paper in (True, False):
+        s = run_case(sh, lp, lq, cfg.dtype, cfg.temperature, un, paper_layout=paper, label="c1")
+        print("c1 paper=%s %r" % (paper, s))
+
+
+def test_config2_full(sh):
+    cfg = workloads.CONFIGS["c2"]
+    lp, lq = workloads.host_logits(cfg)
+    un = workloads.host_uniforms(cfg)
+    s = run_case(sh, lp, lq, cfg.dtype, cfg.temperature, un, paper_layout=False, label="c2")
+    print("c2 %r" % s)
+
+
+def sampled_parity(sh, cfg, n_sample, layouts=(False,), extra_rows=()):
+    """Full-size run on device-generated inputs; oracle on sampled rows (plus `extra_rows`)."""
+    tp, tq = workloads.device_logits(cfg)
+    und = workloads.device_uniforms(cfg)
+    B, N, V = tp.shape
+    rng = np.random.default_rng(cfg.seed + 99)
+    rows = sorted(set(int(r) for r in rng.choice(B * N, size=min(n_sample, B * N), replace=False)) | set(extra_rows))
+    bs, ns = np.array([r // N for r in rows]), np.array([r % N for r in rows])
+    idx_b, idx_n = torch.from_numpy(bs).cuda(), torch.from_numpy(ns).cuda()
+    lp = workloads.to_host_f32(tp[idx_b, idx_n])[:, None, :]
+    lq = workloads.to_host_f32(tq[idx_b, idx_n])[:, None, :]
+    un = und[idx_b, idx_n].cpu().numpy()[:, None, :]
+    total = parity.Stats()
+    for paper in layouts:
+        tree = sh.Tree.heap(N, leaves_sample=paper)
+        kind = workloads.paper_node_kind(N) if paper else None
+        for m in METHODS:
+            d = gpu_draft(sh, m, tq, und, tree, cfg.temperature)
+            out = gpu_verify(sh, m, tp, tq, d["tokens"], und, tree, cfg.temperature)
+            torch.cuda.synchronize()
+            dn = {k: v[idx_b, idx_n].cpu().numpy()[:, None] for k, v in d.items()}
+            st, _ = parity.check_draft(m, lq, cfg.temperature, un, dn, label=cfg.name)
+            tok = dn["tokens"]
+            on = {k: out[k][idx_b, idx_n].cpu().numpy()[:, None] for k in
+                  ("accept_idx", "token", "hub", "beta", "rate", "status")}
+            if kind is None:
+                sv, _ = parity.check_verify(m, lp, lq, cfg.temperature, tok, un, None, on, label=cfg.name)
+            else:
+                sv = parity.Stats()
+                for leafness in (0, 1):
+                    sel = np.nonzero(kind[ns] == leafness)[0]
+                    if len(sel) == 0:
+                        continue
+                    sub = {k: v[sel] for k, v in on.items()}
+                    parity.check_verify(m, lp[sel], lq[sel], cfg.temperature, tok[sel], un[sel],
+                                        np.array([leafness], np.uint8), sub, stats=sv, label=cfg.name)
+            # the walk, for every sequence, against the oracle's walk of the GPU's node outputs
+            full = parity.to_numpy({k: out[k] for k in ("accept_idx", "token", "n_accepted", "n_emitted",
+                                                        "path_nodes", "path_tokens")})
+            w = oracle.walk(full["accept_idx"], full["token"], tree.levels, node_kind=kind)
+            for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+                np.testing.assert_array_equal(full[k], w[k], err_msg=k)
+            # properties that hold at any size
+            st_all = out["status"]
+            assert int((st_all & 3).sum()) == 0
+            assert bool(((out["token"] >= 0) & (out["token"] < V)).all())
+            rate = out["rate"]
+            assert float((rate.sum(-1) - 1).abs().max()) < 1e-4
+            for s in (st, sv):
+                total.rows += s.rows; total.exact += s.exact
+                total.exempt_test += s.exempt_test; total.exempt_token += s.exempt_token
+                total.max_rel = max(total.max_rel, s.max_rel)
+            del d, out
+    del tp, tq
+    torch.cuda.empty_cache()
+    return total
+
+
+@pytest.mark.parametrize("variant", range(4))
+def test_config3_sampled(sh, variant):
+    cfg = workloads.variants("c3")[variant]
+    s = sampled_parity(sh, cfg, 96)
+    print("%s %r" % (cfg.name, s))
+
+
+def test_config4_sampled(sh):
+    cfg = workloads.CONFIGS["c4"]
+    s = sampled_parity(sh, cfg, 64, layouts=(False, True))
+    print("c4 %r" % s)
+
+
+def test_config5_sampled(sh):
+    cfg = workloads.CONFIGS["c5"]
+    if torch.cuda.get_device_properties(0).total_memory < 60e9:
+        pytest.skip("needs ~25 GB of device memory")
+    # make sure every adversarial kind is among the checked rows
+    per_kind = {}
+    for b in range(cfg.batch):
+        for n in range(cfg.nodes):
+            k = workloads._adversarial_kind(cfg, b, n)
+            if k >= 0 and len(per_kind.setdefault(k, [])) < 3:
+                per_kind[k].append(b * cfg.nodes + n)
+    assert len(per_kind) == len(workloads.ADV_KINDS)
+    extra = [(r, k) for k, rows in per_kind.items() for r in rows]
+    s = sampled_parity(sh, cfg, 48, extra_rows=[e[0] for e in extra])
+    print("c5 %r" % s)
