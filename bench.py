@@ -43,6 +43,8 @@ def parse():
     ap.add_argument("--workload", default="c4", choices=sorted(workloads.CONFIGS))
     ap.add_argument("--layout", default="dense", choices=["dense", "paper"],
                     help="dense: every node verifies; paper: last-level nodes only draw the bonus token")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch (profiling on a small case; not a bench value)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle timing leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -184,6 +186,10 @@ def measured_peak():
 def main():
     args = parse()
     cfg = workloads.CONFIGS[args.workload]
+    if args.batch:
+        from dataclasses import replace as _replace
+
+        cfg = _replace(cfg, name=cfg.name + "-batch%d" % args.batch, batch=args.batch)
     if args.impl == "reference":
         run_reference(args, cfg)
         return

@@ -75,6 +75,7 @@ extern "C" {
 #define SPECHUB_ST_DEGENERATE_Q 4u    /* draft mass outside the excluded token is 0 (one-hot q)    */
 #define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
 #define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
+#define SPECHUB_ST_INTERNAL 32u       /* a bounded wait for an on-chip copy expired: row output is -1 */
 
 /* node kinds */
 #define SPECHUB_NODE_VERIFY 0 /* run the accept/reject tests on the node's two drafts         */

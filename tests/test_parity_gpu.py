@@ -108,6 +108,27 @@ def test_small_shapes(sh, V, dtype):
     assert s.rows and s2.rows
 
 
+@pytest.mark.parametrize("V", [4096, 8192, 9000, 12344, 16384, 16392, 24000, 40000, 70000, 81920])
+def test_resident_shapes(sh, V):
+    """bf16, aligned, V % 8 == 0: shapes that take the register-resident cluster kernels
+    (1, 2, 4 CTAs per row; 2, 4 and 5 vectors per thread), with ragged last slices."""
+    rng = np.random.default_rng(V + 3)
+    B, N = 5, 7
+    lp, lq = random_logits(rng, B, N, V, "bf16")
+    # sprinkle the degenerate kinds in
+    lq[0, 1] = lp[0, 1]
+    lq[1, 2] = -np.inf; lq[1, 2, V - 1] = 0.0
+    lq[2, 0] = -60.0; lq[2, 0, V // 2] = 0.0
+    lp[3, 3, : V // 2] = -np.inf; lq[3, 3, V // 2:] = -np.inf
+    lp[4, 4] = np.round(lp[4, 4] * 2) / 2; lq[4, 4] = np.round(lq[4, 4] * 2) / 2
+    lq[4, 5, 7] = lq[4, 5].max() + 9.0   # peaked draft
+    lp, lq = workloads.round_to_storage(lp, "bf16"), workloads.round_to_storage(lq, "bf16")
+    un = random_uniforms(rng, B, N)
+    T = np.array([1.0, 0.6, 1.3, 0.8, 1.0], np.float32)
+    run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="resident-dense")
+    run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="resident-paper")
+
+
 def test_peaked_rows_keep_precision(sh):
     """q close to one-hot: 1 - q(a) must come from a direct sum, not from 1 - q(a)."""
     rng = np.random.default_rng(5)
