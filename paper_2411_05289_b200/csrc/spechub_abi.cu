@@ -6,7 +6,7 @@
 #include "spechub.h"
 #include "spechub_common.cuh"
 #include "spechub_stream.cuh"
-#include "spechub_resident.cuh"
+#include "spechub_lean.cuh"
 
 namespace {
 
@@ -60,66 +60,10 @@ RowArgs base_args(const spechub_desc *d) {
     return a;
 }
 
-// ---- register-resident path ------------------------------------------------------------------------
-// Chosen for bf16 rows with 16-byte aligned starts and V a multiple of 8 when a cluster of C CTAs x
-// 512 threads x NV vectors can hold the row and is at least half full.  Fewer, fatter CTAs per row
-// are preferred: the per-row synchronisation cost is paid once per cluster.
-struct ResPlan {
-    int C, NV, Lc;
-    bool ok;
-};
-
-ResPlan plan_resident(const spechub_desc *d, bool aligned) {
-    ResPlan pl = {0, 0, 0, false};
-    if (d->dtype != SPECHUB_BF16 || !aligned || d->vocab % 8 != 0) return pl;
-    static const int nvs[3] = {2, 4, 5};
-    for (int C = 1; C <= kMaxCluster; C *= 2) {
-        for (int i = 0; i < 3; ++i) {
-            const int NV = nvs[i];
-            const long long cap = (long long)C * kResThreads * NV * 8;
-            if (cap < d->vocab) continue;
-            if (2LL * d->vocab < cap) return pl;  // too small for the smallest fitting shape
-            const int Lc = ((d->vocab + C - 1) / C + 7) / 8 * 8;
-            if ((long long)(C - 1) * Lc >= d->vocab) continue;  // a rank would be empty
-            pl.C = C; pl.NV = NV; pl.Lc = Lc; pl.ok = true;
-            return pl;
-        }
-    }
-    return pl;
-}
-
-template <int NV>
-int launch_resident_spechub(const ResPlan &pl, const ResArgs &ra, cudaStream_t s) {
-    auto kern = resident_spechub_kernel<NV>;
-    constexpr size_t kCtl = (sizeof(ResShared) + 127) / 128 * 128;
-    const size_t smem = kCtl + (size_t)4 * pl.Lc * sizeof(__nv_bfloat16);
-    // one-time function attributes and the number of co-resident clusters, per cluster size
-    static int max_clusters[kMaxCluster + 1] = {0};
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-            return SPECHUB_ERR_LAUNCH;
-        attr_set = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = pl.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    cfg.blockDim = dim3(kResThreads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
-    if (max_clusters[pl.C] == 0) {
-        cfg.gridDim = dim3(pl.C * 64);
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) {
-            (void)cudaGetLastError();
-            return SPECHUB_ERR_LAUNCH;
-        }
-        max_clusters[pl.C] = n;
-    }
-    const int ncl = ra.rows < max_clusters[pl.C] ? ra.rows : max_clusters[pl.C];
-    cfg.gridDim = dim3(ncl * pl.C);
-    ResArgs args = ra;
-    return cudaLaunchKernelEx(&cfg, kern, args) == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+// The lean kernels take bf16 rows whose starts are 16-byte aligned and whose length is a
+// multiple of 8 and large enough to keep 512 threads busy.
+bool lean_ok(const spechub_desc *d, bool aligned) {
+    return d->dtype == SPECHUB_BF16 && aligned && d->vocab % 8 == 0 && d->vocab >= 8192;
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH; }
@@ -142,7 +86,9 @@ int draft_common(const spechub_desc *d, const void *draft_logits, const float *u
     const int th = threads_for(d);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, draft_logits);
-    if (d->dtype == SPECHUB_BF16) {
+    if (lean_ok(d, al)) {
+        lean_draft_kernel<<<rows, kLeanThreads, 0, s>>>(a, method);
+    } else if (d->dtype == SPECHUB_BF16) {
         if (al) draft_rows_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(a, method);
         else draft_rows_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(a, method);
     } else {
@@ -191,15 +137,10 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
     const int th = threads_for(d);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, target_logits) && rows_aligned(d, draft_logits);
-    const ResPlan pl = plan_resident(d, al);
-    if (method == kSpecHub && pl.ok) {
-        ResArgs ra;
-        ra.r = a; ra.rows = (int)rows; ra.Lc = pl.Lc;
-        int rrc = SPECHUB_ERR_LAUNCH;
-        if (pl.NV == 2) rrc = launch_resident_spechub<2>(pl, ra, s);
-        else if (pl.NV == 4) rrc = launch_resident_spechub<4>(pl, ra, s);
-        else rrc = launch_resident_spechub<5>(pl, ra, s);
-        if (rrc != SPECHUB_OK) return rrc;
+    if (lean_ok(d, al)) {
+        if (method == kSpecHub) lean_verify_kernel<kSpecHub><<<rows, kLeanThreads, 0, s>>>(a);
+        else if (method == kRRS) lean_verify_kernel<kRRS><<<rows, kLeanThreads, 0, s>>>(a);
+        else lean_verify_kernel<kRRSw><<<rows, kLeanThreads, 0, s>>>(a);
     } else if (method == kSpecHub) launch_verify<kSpecHub>(d, a, al, rows, th, s);
     else if (method == kRRS) launch_verify<kRRS>(d, a, al, rows, th, s);
     else launch_verify<kRRSw>(d, a, al, rows, th, s);

@@ -1,0 +1,527 @@
+// Lean streaming kernels for bf16 rows with 16-byte aligned starts and V % 8 == 0
+// (the shapes of the large-vocabulary workloads).  One CTA per (sequence, node)
+// row, several CTAs per SM so that one row's reductions overlap another row's
+// streaming.  Compared with the general kernels in spechub_stream.cuh the inner
+// loops are branch-free and carry no index bookkeeping:
+//
+//   pass A  per 16-byte vector: a packed bf16 max tree (4 ops), 8 x (unpack, FMA,
+//           ex2, add).  The exponent reference c of a thread is the maximum of the
+//           first vector it reads, not a running maximum: 2^(k l - c) is exact in
+//           floating point for any c within 2^+-100 of the true one, so c only
+//           moves if a partial sum leaves that range (checked once per vector).
+//   argmax  only threads whose maximum equals the row maximum rescan their own
+//           elements (L2 hits) for the first index; the one owner also re-sums its
+//           elements without the maximum, so 1 - q(a) is a direct sum.
+//   pass B  re-reads the row (L2), recomputes the probabilities and the transport
+//           sums; the hub's pair is removed in the one iteration that holds it.
+//
+// The special-function pipe (16 ex2/clk/SM) bounds both passes: 4 ex2 per
+// vocabulary pair per row.
+#pragma once
+
+#include "spechub.h"
+#include "spechub_common.cuh"
+#include "spechub_stream.cuh"
+
+namespace spechub {
+
+constexpr int kLeanThreads = 512;
+constexpr int kLeanWarps = kLeanThreads / 32;
+constexpr float kHuge = 1.0e30f;  // ~2^100: partial sums beyond this move the reference
+
+struct LeanShared {
+    float wml[2][kLeanWarps];    // per-warp max logit (0 target, 1 draft)
+    float wmass[2][kLeanWarps];  // per-warp sum of exponentials on the row's scale, argmax left out
+    int cand[2];                 // lowest index attaining the row maximum
+    float acc[4][kLeanWarps];
+    float mass[kLeanWarps];
+    int tok;
+};
+
+__device__ __forceinline__ unsigned bf2max(unsigned a, unsigned b) {
+    unsigned d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ float bf2_hmax(unsigned m2) {
+    return fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+}
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float (&o)[8]) {
+    o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+    o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+    o[4] = __uint_as_float(v.z << 16); o[5] = __uint_as_float(v.z & 0xffff0000u);
+    o[6] = __uint_as_float(v.w << 16); o[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+struct LeanAcc {  // one thread's pass-A state for one row
+    unsigned m2;  // packed running maximum
+    float c;      // exponent reference (k * some logit of this thread, or 0)
+    float s;      // sum of 2^(k l - c)
+};
+
+__device__ __forceinline__ void lean_push(LeanAcc &st, const uint4 &raw, float k) {
+    const unsigned vm = bf2max(bf2max(raw.x, raw.y), bf2max(raw.z, raw.w));
+    st.m2 = bf2max(st.m2, vm);
+    float v[8];
+    unpack_bf16x8(raw, v);
+    float e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) e[i] = ex2(__fmaf_rn(v[i], k, -st.c));
+    float a = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    if (!(a < kHuge)) {  // out of range (or NaN / +inf input): move the reference to this vector's max
+        const float vmax = bf2_hmax(vm);
+        const float cn = shift_of(vmax, k);
+        st.s *= ex2(st.c - cn);
+        st.c = cn;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) e[i] = ex2(__fmaf_rn(v[i], k, -st.c));
+        a = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    }
+    st.s += a;
+}
+
+// Pass A over this warp's range of one or two rows.
+template <bool BOTH>
+__device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, int lo, int hi, int lane,
+                                            float k, LeanAcc &P, LeanAcc &Q) {
+    P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
+    Q.m2 = 0xff80ff80u; Q.s = 0.f; Q.c = 0.f;
+    int vi = lo + lane;
+    // the reference comes from the thread's first vector that holds a finite logit
+    for (int vr = vi; vr < hi; vr += 32) {
+        const uint4 a = rp[vr];
+        const float m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
+        if (m0 > neg_inf()) { P.c = shift_of(m0, k); break; }
+    }
+    if (BOTH) {
+        for (int vr = vi; vr < hi; vr += 32) {
+            const uint4 b = rq[vr];
+            const float m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
+            if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
+        }
+    }
+#pragma unroll 2
+    for (; vi < hi; vi += 32) {
+        const uint4 a = rp[vi];
+        uint4 b;
+        if (BOTH) b = rq[vi];
+        lean_push(P, a, k);
+        if (BOTH) lean_push(Q, b, k);
+    }
+}
+
+// A thread whose maximum equals the row maximum `val` rescans its elements: first index of val,
+// and the sum of 2^(k l - c) over its elements without that index (same order as pass A).
+__device__ __forceinline__ void lean_rescan(const uint4 *row, int lo, int hi, int lane, float val, float k,
+                                            float c, int &first_idx, float &s_excl) {
+    first_idx = 0x7fffffff;
+    float s = 0.f;
+    for (int vi = lo + lane; vi < hi; vi += 32) {
+        float v[8];
+        unpack_bf16x8(row[vi], v);
+        float e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool hit = (v[i] == val) && first_idx == 0x7fffffff;
+            if (hit) first_idx = vi * 8 + i;
+            e[i] = hit ? 0.f : ex2(__fmaf_rn(v[i], k, -c));
+        }
+        s += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    }
+    s_excl = s;
+}
+
+// Row-level (max, argmax, sum without the argmax) from the per-thread pass-A states.
+// Leaves the per-warp masses (row scale, argmax left out) in sh.wmass[r] for the samplers.
+// All threads call it; r = 0 target, 1 draft.
+__device__ ArgMaxSum lean_reduce(const LeanAcc &st, const uint4 *row, int lo, int hi, float k, int r,
+                                 LeanShared &sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float ml = bf2_hmax(st.m2);
+    float wm = ml;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(kFull, wm, o));
+    if (lane == 0) sh.wml[r][warp] = wm;
+    if (threadIdx.x == 0) sh.cand[r] = 0x7fffffff;
+    __syncthreads();
+    float rm = sh.wml[r][0];
+#pragma unroll
+    for (int w = 1; w < kLeanWarps; ++w) rm = fmaxf(rm, sh.wml[r][w]);
+    int myidx = 0x7fffffff;
+    float sx = 0.f;
+    const bool cand = (ml == rm) && rm > neg_inf() && rm < -neg_inf();
+    if (cand) {
+        lean_rescan(row, lo, hi, lane, rm, k, st.c, myidx, sx);
+        atomicMin(&sh.cand[r], myidx);
+    }
+    __syncthreads();
+    const int idx = sh.cand[r];
+    const float C = shift_of(rm, k);
+    const float mine = (cand && myidx == idx) ? sx : st.s;
+    // threads whose reference is still 0 with nothing finite seen carry no mass
+    float v = mine * ex2(st.c - C);
+    if (!(ml > neg_inf())) v = 0.f;
+    v = warp_sum(v);
+    if (lane == 0) sh.wmass[r][warp] = v;
+    __syncthreads();
+    ArgMaxSum out;
+    out.ml = rm; out.c = C; out.idx = idx;
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kLeanWarps; ++w) t += sh.wmass[r][w];
+    out.sx = t;
+    return out;
+}
+
+// Draw from softmax(row), with token `excl` removed (excl < 0: none).  `hubtok` is the row's
+// argmax, whose exponential sh.wmass leaves out.
+__device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, float C, int hubtok,
+                               int excl, float u, int r, LeanShared &sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x < kLeanWarps) {
+        const int w = threadIdx.x;
+        const bool holds_hub = (hubtok / 8) >= g.seg_lo(w) && (hubtok / 8) < g.seg_hi(w);
+        sh.mass[w] = sh.wmass[r][w] + ((holds_hub && excl != hubtok) ? 1.f : 0.f);
+    }
+    __syncthreads();
+    if (excl >= 0 && excl != hubtok) {
+        const int wex = (excl / 8) / g.seg;
+        if (warp == wex) {
+            float s = 0.f;
+            for (int vi = g.seg_lo(warp) + lane; vi < g.seg_hi(warp); vi += 32) {
+                float v[8];
+                load_vec<__nv_bfloat16, true>(row, vi, g.V, v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) s += (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
+            }
+            s = warp_sum(s);
+            if (lane == 0) sh.mass[warp] = s;
+        }
+        __syncthreads();
+    }
+    auto wf = [&](int vi, float(&w)[8]) {
+        float v[8];
+        load_vec<__nv_bfloat16, true>(row, vi, g.V, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
+    };
+    return block_sample<8>(g, wf, sh.mass, u, &sh.tok);
+}
+
+template <int NACC>
+__device__ __forceinline__ void lean_block_sums(float (&x)[NACC], LeanShared &sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int i = 0; i < NACC; ++i) {
+        const float s = warp_sum(x[i]);
+        if (lane == 0) sh.acc[i][warp] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < NACC; ++i) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kLeanWarps; ++w) t += sh.acc[i][w];
+        x[i] = t;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
+// ------------------------------------------------------------------------------------------------
+template <int METHOD>
+__global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a) {
+    __shared__ LeanShared sh;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    const __nv_bfloat16 *rowp = static_cast<const __nv_bfloat16 *>(a.target) + b * a.stride_seq + n * a.stride_node;
+    const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(rowp), *vq = reinterpret_cast<const uint4 *>(rowq);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const float k = kLog2e / temperature_of(a, b);
+    const float r1 = a.uniforms[r * 5 + 2], r2 = a.uniforms[r * 5 + 3], ures = a.uniforms[r * 5 + 4];
+    const float pinf = -neg_inf();
+    const bool leaf = a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF;
+
+    NodeResult o;
+    o.accept_idx = -1; o.token = -1; o.hub = -1; o.status = 0;
+    o.beta[0] = o.beta[1] = 0.f; o.rate[0] = o.rate[1] = o.rate[2] = 0.f;
+
+    LeanAcc tp, tq;
+    if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
+    else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
+    const ArgMaxSum P = lean_reduce(tp, vp, lo, hi, k, 0, sh);
+    const float Zp = P.sx + 1.f;
+    if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
+        o.status = SPECHUB_ST_NONFINITE;
+        if (threadIdx.x == 0) write_node(a, r, o);
+        return;
+    }
+    const float cP = P.c, invZp = 1.f / Zp;
+    if (leaf) {
+        o.token = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
+        o.rate[2] = 1.f;
+        if (threadIdx.x == 0) write_node(a, r, o);
+        return;
+    }
+    const ArgMaxSum Q = lean_reduce(tq, vq, lo, hi, k, 1, sh);
+    const float Zq = Q.sx + 1.f;
+    if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) {
+        o.status = SPECHUB_ST_NONFINITE;
+        if (threadIdx.x == 0) write_node(a, r, o);
+        return;
+    }
+    const float cQ = Q.c, invZq = 1.f / Zq;
+    const int x1 = a.draft_tokens_in[2 * r], x2 = a.draft_tokens_in[2 * r + 1];
+    auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
+    auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
+
+    if (METHOD == kSpecHub) {
+        const int hubtok = Q.idx;
+        o.hub = hubtok;
+        const bool pair_xa = (x2 == hubtok && x1 != hubtok), pair_ax = (x1 == hubtok && x2 != hubtok);
+        const int x = pair_xa ? x1 : x2;
+        if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) {
+            o.status = SPECHUB_ST_TOKEN_RANGE;
+            if (threadIdx.x == 0) write_node(a, r, o);
+            return;
+        }
+        const bool degenerate = !(Q.sx > 0.f);
+        const float c = degenerate ? 0.f : 1.f / Q.sx;
+        const float qa = invZq, rest = Q.sx * invZq;
+        const int hubvec = hubtok >> 3, hubel = hubtok & 7;
+        // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
+        float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
+#pragma unroll 2
+        for (int vi = lo + lane; vi < hi; vi += 32) {
+            float fp[8], fq[8];
+            unpack_bf16x8(vp[vi], fp);
+            unpack_bf16x8(vq[vi], fq);
+            if (vi == hubvec) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i == hubel) { fp[i] = neg_inf(); fq[i] = neg_inf(); }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {
+                float d, t;
+                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
+                transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), c, d, t);
+                s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
+            }
+        }
+        float acc[3] = {s1a + s1b, s2a + s2b, ra + rb};
+        lean_block_sums<3>(acc, sh);
+        const float S1 = acc[0], S2 = degenerate ? qa : acc[1], R = acc[2];
+        const float pa = prob_p(hubtok);
+        const float hub_left = fmaxf(pa - S2, 0.f);
+        o.rate[0] = fmaxf(rest - S1, 0.f) + fminf(pa, S2);
+        o.rate[1] = (degenerate ? 0.f : fmaxf(qa - S2, 0.f)) + fminf(hub_left, S1);
+        o.rate[2] = R;
+        if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
+        const float px = prob_p(x), qx = prob_q(x);
+        bool acc1, acc2;
+        if (pair_xa) {
+            acc1 = accept_test(r1, px, qx, o.beta[0], true, o.status);
+            if (acc1) { o.accept_idx = 0; o.token = x; }
+            acc2 = accept_test(r2, hub_left, S1, o.beta[1], !acc1, o.status);
+            if (!acc1 && acc2) { o.accept_idx = 1; o.token = hubtok; }
+        } else {
+            acc1 = accept_test(r1, fmaxf(__fsub_rn(px, qx), 0.f), c * qx, o.beta[0], true, o.status);
+            if (acc1) { o.accept_idx = 1; o.token = x; }
+            acc2 = accept_test(r2, pa, S2, o.beta[1], !acc1, o.status);
+            if (!acc1 && acc2) { o.accept_idx = 0; o.token = hubtok; }
+        }
+        if (!(acc1 || acc2)) {
+            if (threadIdx.x < kLeanWarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
+            __syncthreads();
+            auto wf = [&](int vi, float(&w)[8]) {
+                float fp[8], fq[8];
+                unpack_bf16x8(vp[vi], fp);
+                unpack_bf16x8(vq[vi], fq);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float d, t;
+                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                    w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
+                }
+            };
+            int tok = block_sample<8>(g, wf, sh.mass, ures, &sh.tok);
+            if (tok < 0) {
+                o.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
+            }
+            o.accept_idx = -1;
+            o.token = tok;
+        }
+    } else {
+        if (x1 < 0 || x1 >= a.vocab || x2 < 0 || x2 >= a.vocab) {
+            o.status = SPECHUB_ST_TOKEN_RANGE;
+            if (threadIdx.x == 0) write_node(a, r, o);
+            return;
+        }
+        // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
+        const int x1vec = x1 >> 3, x1el = x1 & 7;
+        float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
+#pragma unroll 2
+        for (int vi = lo + lane; vi < hi; vi += 32) {
+            float fp[8], fq[8];
+            unpack_bf16x8(vp[vi], fp);
+            unpack_bf16x8(vq[vi], fq);
+            float pp[8], qq[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {
+                a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
+                a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
+            }
+            if (METHOD == kRRSw) {
+                if (vi == x1vec) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i == x1el) qq[i] = 0.f;
+                }
+                dna += (qq[0] + qq[1]) + (qq[2] + qq[3]);
+                dnb += (qq[4] + qq[5]) + (qq[6] + qq[7]);
+            }
+        }
+        float acc[2] = {a1a + a1b, dna + dnb};
+        lean_block_sums<2>(acc, sh);
+        release_sums();
+        const float A1 = acc[0], den = acc[1];
+        const bool q1_zero = (METHOD == kRRSw) && !(den > 0.f);
+        const float gq = (METHOD == kRRSw) ? (q1_zero ? 0.f : 1.f / den) : 1.f;
+        const float A1g = A1 * gq;
+        // pass C: mass of the residual after two rejections
+        float w2a = 0.f, w2b = 0.f;
+#pragma unroll 2
+        for (int vi = lo + lane; vi < hi; vi += 32) {
+            float fp[8], fq[8];
+            unpack_bf16x8(vp[vi], fp);
+            unpack_bf16x8(vq[vi], fq);
+            float sc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sc[i] = A1g;
+            if (METHOD == kRRSw && vi == x1vec) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i == x1el) sc[i] = 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {
+                float d, t;
+                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc[i], d, t);
+                w2a += fmaxf(t, 0.f);
+                transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), sc[i + 1], d, t);
+                w2b += fmaxf(t, 0.f);
+            }
+        }
+        float w2[1] = {w2a + w2b};
+        lean_block_sums<1>(w2, sh);
+        const float W2 = w2[0];
+        o.rate[0] = fmaxf(1.f - A1, 0.f);
+        o.rate[1] = fmaxf(A1 - W2, 0.f);
+        o.rate[2] = W2;
+        const float px1 = prob_p(x1), qx1 = prob_q(x1), px2 = prob_p(x2), qx2 = prob_q(x2);
+        const bool acc1 = accept_test(r1, px1, qx1, o.beta[0], true, o.status);
+        if (acc1) { o.accept_idx = 0; o.token = x1; }
+        if (!acc1 && q1_zero) o.status |= SPECHUB_ST_DEGENERATE_Q;
+        bool acc2 = false;
+        if (A1 > 0.f) {
+            const float q1x2 = (METHOD == kRRSw && x2 == x1) ? 0.f : A1g * qx2;
+            acc2 = accept_test(r2, fmaxf(__fsub_rn(px2, qx2), 0.f), q1x2, o.beta[1], !acc1, o.status);
+        }
+        if (!acc1 && acc2) { o.accept_idx = 1; o.token = x2; }
+        if (!(acc1 || acc2)) {
+            int tok = -1;
+            if (A1 > 0.f) {
+                if (threadIdx.x < kLeanWarps) sh.mass[threadIdx.x] = sh.acc[0][threadIdx.x];
+                __syncthreads();
+                auto wf = [&](int vi, float(&w)[8]) {
+                    float fp[8], fq[8];
+                    unpack_bf16x8(vp[vi], fp);
+                    unpack_bf16x8(vq[vi], fq);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float d, t;
+                        const float s = (METHOD == kRRSw && vi * 8 + i == x1) ? 0.f : A1g;
+                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), s, d, t);
+                        w[i] = fmaxf(t, 0.f);
+                    }
+                };
+                tok = block_sample<8>(g, wf, sh.mass, ures, &sh.tok);
+            }
+            if (tok < 0) {
+                o.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
+            }
+            o.accept_idx = -1;
+            o.token = tok;
+        }
+    }
+    if (threadIdx.x == 0) write_node(a, r, o);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Draft step.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kLeanThreads, 2) lean_draft_kernel(RowArgs a, int method) {
+    __shared__ LeanShared sh;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vq = reinterpret_cast<const uint4 *>(rowq);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const float k = kLog2e / temperature_of(a, b);
+    const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
+
+    LeanAcc tq, unused;
+    lean_pass_a<false>(vq, vq, lo, hi, lane, k, tq, unused);
+    const ArgMaxSum q = lean_reduce(tq, vq, lo, hi, k, 1, sh);
+    const float Zq = q.sx + 1.f;
+    uint32_t st = 0;
+    int x1 = -1, x2 = -1, hubtok = -1;
+    float prob0 = 0.f, prob1 = 0.f;
+    if (!(q.ml > neg_inf()) || !finite_pos(Zq) || !(q.ml < -neg_inf())) {
+        st = SPECHUB_ST_NONFINITE;
+    } else {
+        hubtok = q.idx;
+        x1 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u1, 1, sh);
+        if (method == kSpecHub) {
+            prob0 = 1.f / Zq;
+            if (x1 != hubtok) {
+                x2 = hubtok;
+                prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -q.c)) / Zq;
+            } else if (!(q.sx > 0.f)) {
+                x2 = (hubtok == 0) ? 1 : 0;
+                st |= SPECHUB_ST_DEGENERATE_Q;
+            } else {
+                x2 = lean_sample_row(g, rowq, k, q.c, hubtok, hubtok, u2, 1, sh);
+                prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2), k, -q.c)) / q.sx;
+            }
+        } else if (method == kRRS) {
+            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u2, 1, sh);
+        } else {
+            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, x1, u2, 1, sh);
+            if (x2 < 0) {
+                x2 = (x1 == 0) ? 1 : 0;
+                st |= SPECHUB_ST_DEGENERATE_Q;
+            }
+        }
+    }
+    if (threadIdx.x == 0) {
+        a.draft_tokens_out[2 * r] = x1;
+        a.draft_tokens_out[2 * r + 1] = x2;
+        if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;
+        if (a.draft_prob) { a.draft_prob[2 * r] = prob0; a.draft_prob[2 * r + 1] = prob1; }
+        if (a.status) a.status[r] = st;
+    }
+}
+
+}  // namespace spechub

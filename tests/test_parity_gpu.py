@@ -109,9 +109,9 @@ def test_small_shapes(sh, V, dtype):
 
 
 @pytest.mark.parametrize("V", [4096, 8192, 9000, 12344, 16384, 16392, 24000, 40000, 70000, 81920])
-def test_resident_shapes(sh, V):
-    """bf16, aligned, V % 8 == 0: shapes that take the register-resident cluster kernels
-    (1, 2, 4 CTAs per row; 2, 4 and 5 vectors per thread), with ragged last slices."""
+def test_lean_shapes(sh, V):
+    """bf16, aligned, V % 8 == 0: shapes that take the lean bf16 kernels (V >= 8192) or, below that, the general ones
+    with ragged warp ranges."""
     rng = np.random.default_rng(V + 3)
     B, N = 5, 7
     lp, lq = random_logits(rng, B, N, V, "bf16")
@@ -125,8 +125,8 @@ def test_resident_shapes(sh, V):
     lp, lq = workloads.round_to_storage(lp, "bf16"), workloads.round_to_storage(lq, "bf16")
     un = random_uniforms(rng, B, N)
     T = np.array([1.0, 0.6, 1.3, 0.8, 1.0], np.float32)
-    run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="resident-dense")
-    run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="resident-paper")
+    run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="lean-dense")
+    run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="lean-paper")
 
 
 def test_peaked_rows_keep_precision(sh):
