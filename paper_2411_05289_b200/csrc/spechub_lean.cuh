@@ -25,16 +25,15 @@
 
 namespace spechub {
 
-constexpr int kLeanThreads = 512;
-constexpr int kLeanWarps = kLeanThreads / 32;
+constexpr int kLeanMaxWarps = 32;
 constexpr float kHuge = 1.0e30f;  // ~2^100: partial sums beyond this move the reference
 
 struct LeanShared {
-    float wml[2][kLeanWarps];    // per-warp max logit (0 target, 1 draft)
-    float wmass[2][kLeanWarps];  // per-warp sum of exponentials on the row's scale, argmax left out
-    int cand[2];                 // lowest index attaining the row maximum
-    float acc[4][kLeanWarps];
-    float mass[kLeanWarps];
+    float wml[2][kLeanMaxWarps];    // per-warp max logit (0 target, 1 draft)
+    float wmass[2][kLeanMaxWarps];  // per-warp sum of exponentials on the row's scale, argmax left out
+    int cand[2];                    // lowest index attaining the row maximum
+    float acc[4][kLeanMaxWarps];
+    float mass[kLeanMaxWarps];
     int tok;
 };
 
@@ -110,67 +109,213 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
     }
 }
 
-// A thread whose maximum equals the row maximum `val` rescans its elements: first index of val,
-// and the sum of 2^(k l - c) over its elements without that index (same order as pass A).
-__device__ __forceinline__ void lean_rescan(const uint4 *row, int lo, int hi, int lane, float val, float k,
-                                            float c, int &first_idx, float &s_excl) {
-    first_idx = 0x7fffffff;
-    float s = 0.f;
-    for (int vi = lo + lane; vi < hi; vi += 32) {
+// The lanes of a warp rescan, together, the elements of its lane `src` (whose maximum equals the
+// row maximum `val`): lane j takes the j-th vector of that thread, so the rescan costs one load
+// round trip instead of one per vector.  Returns (to every lane) the first index of val among
+// those elements and the sum of 2^(k l - c) over them without that index.
+__device__ __forceinline__ void lean_rescan_warp(const uint4 *row, int lo, int hi, int lane, int src,
+                                                 float val, float k, float c, int &first_idx,
+                                                 float &s_excl) {
+    int fi = 0x7fffffff;
+    // pass 1: first index
+    for (int vj = lo + src + 32 * lane; vj < hi; vj += 32 * 32) {
         float v[8];
-        unpack_bf16x8(row[vi], v);
+        unpack_bf16x8(row[vj], v);
+#pragma unroll
+        for (int i = 7; i >= 0; --i)
+            if (v[i] == val) fi = min(fi, vj * 8 + i);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) fi = min(fi, __shfl_xor_sync(kFull, fi, o));
+    // pass 2: the sum without it (the vectors are L1/L2 hits now)
+    float s = 0.f;
+    for (int vj = lo + src + 32 * lane; vj < hi; vj += 32 * 32) {
+        float v[8];
+        unpack_bf16x8(row[vj], v);
         float e[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const bool hit = (v[i] == val) && first_idx == 0x7fffffff;
-            if (hit) first_idx = vi * 8 + i;
-            e[i] = hit ? 0.f : ex2(__fmaf_rn(v[i], k, -c));
-        }
+        for (int i = 0; i < 8; ++i) e[i] = (vj * 8 + i == fi) ? 0.f : ex2(__fmaf_rn(v[i], k, -c));
         s += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
     }
-    s_excl = s;
+    s_excl = warp_sum(s);
+    first_idx = fi;
 }
 
-// Row-level (max, argmax, sum without the argmax) from the per-thread pass-A states.
-// Leaves the per-warp masses (row scale, argmax left out) in sh.wmass[r] for the samplers.
-// All threads call it; r = 0 target, 1 draft.
-__device__ ArgMaxSum lean_reduce(const LeanAcc &st, const uint4 *row, int lo, int hi, float k, int r,
-                                 LeanShared &sh) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float ml = bf2_hmax(st.m2);
-    float wm = ml;
+// Row-level (max, argmax, sum without the argmax) of the target (r = 0) and, if BOTH, the draft
+// (r = 1) from the per-thread pass-A states.  Leaves the per-warp masses (row scale, argmax left
+// out) in sh.wmass[r] for the samplers.  All threads call it.
+template <bool BOTH>
+__device__ void lean_reduce2(const LeanAcc &tp, const LeanAcc &tq, const uint4 *vp, const uint4 *vq, int lo,
+                             int hi, float k, LeanShared &sh, ArgMaxSum &P, ArgMaxSum &Q) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const float mlp = bf2_hmax(tp.m2), mlq = BOTH ? bf2_hmax(tq.m2) : neg_inf();
+    float wp = mlp, wq = mlq;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(kFull, wm, o));
-    if (lane == 0) sh.wml[r][warp] = wm;
-    if (threadIdx.x == 0) sh.cand[r] = 0x7fffffff;
+    for (int o = 16; o > 0; o >>= 1) {
+        wp = fmaxf(wp, __shfl_xor_sync(kFull, wp, o));
+        if (BOTH) wq = fmaxf(wq, __shfl_xor_sync(kFull, wq, o));
+    }
+    if (lane == 0) { sh.wml[0][warp] = wp; sh.wml[1][warp] = wq; }
+    if (threadIdx.x == 0) { sh.cand[0] = 0x7fffffff; sh.cand[1] = 0x7fffffff; }
     __syncthreads();
-    float rm = sh.wml[r][0];
-#pragma unroll
-    for (int w = 1; w < kLeanWarps; ++w) rm = fmaxf(rm, sh.wml[r][w]);
-    int myidx = 0x7fffffff;
-    float sx = 0.f;
-    const bool cand = (ml == rm) && rm > neg_inf() && rm < -neg_inf();
-    if (cand) {
-        lean_rescan(row, lo, hi, lane, rm, k, st.c, myidx, sx);
-        atomicMin(&sh.cand[r], myidx);
+    float rmp = sh.wml[0][0], rmq = sh.wml[1][0];
+    for (int w = 1; w < nwarps; ++w) { rmp = fmaxf(rmp, sh.wml[0][w]); rmq = fmaxf(rmq, sh.wml[1][w]); }
+    const float pinf = -neg_inf();
+    int idxp_mine = 0x7fffffff, idxq_mine = 0x7fffffff;
+    float sxp = 0.f, sxq = 0.f;
+    {
+        const bool cand = (mlp == rmp) && rmp > neg_inf() && rmp < pinf;
+        unsigned cm = __ballot_sync(kFull, cand);
+        while (cm) {
+            const int src = __ffs(cm) - 1;
+            cm &= cm - 1;
+            int fi; float sx;
+            lean_rescan_warp(vp, lo, hi, lane, src, rmp, k, __shfl_sync(kFull, tp.c, src), fi, sx);
+            if (lane == src) { idxp_mine = fi; sxp = sx; atomicMin(&sh.cand[0], fi); }
+        }
+    }
+    if (BOTH) {
+        const bool cand = (mlq == rmq) && rmq > neg_inf() && rmq < pinf;
+        unsigned cm = __ballot_sync(kFull, cand);
+        while (cm) {
+            const int src = __ffs(cm) - 1;
+            cm &= cm - 1;
+            int fi; float sx;
+            lean_rescan_warp(vq, lo, hi, lane, src, rmq, k, __shfl_sync(kFull, tq.c, src), fi, sx);
+            if (lane == src) { idxq_mine = fi; sxq = sx; atomicMin(&sh.cand[1], fi); }
+        }
     }
     __syncthreads();
-    const int idx = sh.cand[r];
-    const float C = shift_of(rm, k);
-    const float mine = (cand && myidx == idx) ? sx : st.s;
-    // threads whose reference is still 0 with nothing finite seen carry no mass
-    float v = mine * ex2(st.c - C);
-    if (!(ml > neg_inf())) v = 0.f;
-    v = warp_sum(v);
-    if (lane == 0) sh.wmass[r][warp] = v;
+    const int idxp = sh.cand[0], idxq = sh.cand[1];
+    const float Cp = shift_of(rmp, k), Cq = shift_of(rmq, k);
+    {
+        const float mine = (idxp_mine != 0x7fffffff && idxp_mine == idxp) ? sxp : tp.s;
+        float v = (mlp > neg_inf()) ? mine * ex2(tp.c - Cp) : 0.f;
+        v = warp_sum(v);
+        if (lane == 0) sh.wmass[0][warp] = v;
+    }
+    if (BOTH) {
+        const float mine = (idxq_mine != 0x7fffffff && idxq_mine == idxq) ? sxq : tq.s;
+        float v = (mlq > neg_inf()) ? mine * ex2(tq.c - Cq) : 0.f;
+        v = warp_sum(v);
+        if (lane == 0) sh.wmass[1][warp] = v;
+    }
     __syncthreads();
-    ArgMaxSum out;
-    out.ml = rm; out.c = C; out.idx = idx;
-    float t = 0.f;
+    float t0 = 0.f, t1 = 0.f;
+    for (int w = 0; w < nwarps; ++w) { t0 += sh.wmass[0][w]; if (BOTH) t1 += sh.wmass[1][w]; }
+    P.ml = rmp; P.c = Cp; P.idx = idxp; P.sx = t0;
+    Q.ml = rmq; Q.c = Cq; Q.idx = idxq; Q.sx = t1;
+}
+
+// CTA-wide inverse-CDF draw with two rounds of warp-parallel loads.  mass[w] (shared) = total
+// weight of warp w's range; weights(vi, w[8]) the weights of vector vi.  In the selected warp,
+// round 1 gives every lane a contiguous block of the range (one scan finds the block), round 2
+// spreads that block's vectors over the lanes (one scan finds the vector).  Same result rule as
+// block_sample.  Must be called by all threads of the CTA.
+template <class WF>
+__device__ int block_sample2(const Geo &g, WF weights, const float *mass, float u, int *sh_tok) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float total = 0.f;
+    for (int w = 0; w < g.nwarps; ++w) total += mass[w];
+    if (!(total > 0.f)) return -1;
+    const float t = u * total;
+    int wsel = -1, lastw = -1;
+    float base = 0.f, lastbase = 0.f, run = 0.f;
+    for (int w = 0; w < g.nwarps; ++w) {
+        const float m = mass[w];
+        if (m > 0.f) {
+            lastw = w;
+            lastbase = run;
+            if (wsel < 0 && run + m > t) { wsel = w; base = run; }
+        }
+        run += m;
+    }
+    if (wsel < 0) { wsel = lastw; base = lastbase; }
+    if (warp == wsel) {
+        const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+        const int J = (hi - lo + 31) / 32;  // vectors per lane block
+        float tt = t - base;
+        // round 1: lane totals over contiguous blocks
+        const int b0 = lo + lane * J, b1 = min(hi, b0 + J);
+        float tot = 0.f;
+#pragma unroll 4
+        for (int vi = b0; vi < b1; ++vi) {
+            float w[8];
+            weights(vi, w);
+            tot += ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+        }
+        float incl = tot;
 #pragma unroll
-    for (int w = 0; w < kLeanWarps; ++w) t += sh.wmass[r][w];
-    out.sx = t;
-    return out;
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const unsigned pos = __ballot_sync(kFull, tot > 0.f);
+        const unsigned hit = __ballot_sync(kFull, tot > 0.f && incl > tt);
+        int found = -1;
+        if (pos) {
+            const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
+            tt -= __shfl_sync(kFull, incl - tot, L);
+            const int c0 = lo + L * J, c1 = min(hi, c0 + J);
+            // round 2: the block's vectors over the lanes
+            float prefix = 0.f;
+            int lastpos = -1;
+            for (int v0 = c0; v0 < c1 && found < 0; v0 += 32) {
+                const int vi = v0 + lane;
+                float w[8];
+                if (vi < c1) {
+                    weights(vi, w);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) w[i] = 0.f;
+                }
+                float lsum = 0.f;
+                int lp = -1;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    lsum += w[i];
+                    if (w[i] > 0.f) lp = vi * 8 + i;
+                }
+                float in2 = lsum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float up = __shfl_up_sync(kFull, in2, o);
+                    if (lane >= o) in2 += up;
+                }
+                const float tot2 = __shfl_sync(kFull, in2, 31);
+                const unsigned hit2 = __ballot_sync(kFull, lsum > 0.f && prefix + in2 > tt);
+                if (hit2) {
+                    const int M = __ffs(hit2) - 1;
+                    int cand = -1;
+                    if (lane == M) {
+                        float acc = prefix + (in2 - lsum);
+                        int lastin = -1;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            acc += w[i];
+                            if (w[i] > 0.f) {
+                                lastin = vi * 8 + i;
+                                if (cand < 0 && acc > tt) cand = lastin;
+                            }
+                        }
+                        if (cand < 0) cand = lastin;
+                    }
+                    found = __shfl_sync(kFull, cand, M);
+                } else {
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(kFull, lp, o));
+                    lastpos = max(lastpos, lp);
+                    prefix += tot2;
+                }
+            }
+            if (found < 0) found = lastpos;
+        }
+        if (lane == 0) *sh_tok = found;
+    }
+    __syncthreads();
+    const int tok = *sh_tok;
+    __syncthreads();
+    return tok;
 }
 
 // Draw from softmax(row), with token `excl` removed (excl < 0: none).  `hubtok` is the row's
@@ -178,7 +323,7 @@ __device__ ArgMaxSum lean_reduce(const LeanAcc &st, const uint4 *row, int lo, in
 __device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, float C, int hubtok,
                                int excl, float u, int r, LeanShared &sh) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x < kLeanWarps) {
+    if (threadIdx.x < g.nwarps) {
         const int w = threadIdx.x;
         const bool holds_hub = (hubtok / 8) >= g.seg_lo(w) && (hubtok / 8) < g.seg_hi(w);
         sh.mass[w] = sh.wmass[r][w] + ((holds_hub && excl != hubtok) ? 1.f : 0.f);
@@ -205,7 +350,7 @@ __device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, 
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
     };
-    return block_sample<8>(g, wf, sh.mass, u, &sh.tok);
+    return block_sample2(g, wf, sh.mass, u, &sh.tok);
 }
 
 template <int NACC>
@@ -217,11 +362,11 @@ __device__ __forceinline__ void lean_block_sums(float (&x)[NACC], LeanShared &sh
         if (lane == 0) sh.acc[i][warp] = s;
     }
     __syncthreads();
+    const int nwarps = blockDim.x >> 5;
 #pragma unroll
     for (int i = 0; i < NACC; ++i) {
         float t = 0.f;
-#pragma unroll
-        for (int w = 0; w < kLeanWarps; ++w) t += sh.acc[i][w];
+        for (int w = 0; w < nwarps; ++w) t += sh.acc[i][w];
         x[i] = t;
     }
 }
@@ -229,8 +374,8 @@ __device__ __forceinline__ void lean_block_sums(float (&x)[NACC], LeanShared &sh
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
-template <int METHOD>
-__global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a) {
+template <int METHOD, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(RowArgs a) {
     __shared__ LeanShared sh;
     const long long r = blockIdx.x;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
@@ -252,7 +397,9 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
     LeanAcc tp, tq;
     if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
-    const ArgMaxSum P = lean_reduce(tp, vp, lo, hi, k, 0, sh);
+    ArgMaxSum P, Q;
+    if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, P, Q);
+    else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, P, Q);
     const float Zp = P.sx + 1.f;
     if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
         o.status = SPECHUB_ST_NONFINITE;
@@ -266,7 +413,6 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
         if (threadIdx.x == 0) write_node(a, r, o);
         return;
     }
-    const ArgMaxSum Q = lean_reduce(tq, vq, lo, hi, k, 1, sh);
     const float Zq = Q.sx + 1.f;
     if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) {
         o.status = SPECHUB_ST_NONFINITE;
@@ -336,7 +482,7 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
             if (!acc1 && acc2) { o.accept_idx = 0; o.token = hubtok; }
         }
         if (!(acc1 || acc2)) {
-            if (threadIdx.x < kLeanWarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
+            if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
             __syncthreads();
             auto wf = [&](int vi, float(&w)[8]) {
                 float fp[8], fq[8];
@@ -349,7 +495,7 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
                     w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
                 }
             };
-            int tok = block_sample<8>(g, wf, sh.mass, ures, &sh.tok);
+            int tok = block_sample2(g, wf, sh.mass, ures, &sh.tok);
             if (tok < 0) {
                 o.status |= SPECHUB_ST_ZERO_RESIDUAL;
                 tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
@@ -439,7 +585,7 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
         if (!(acc1 || acc2)) {
             int tok = -1;
             if (A1 > 0.f) {
-                if (threadIdx.x < kLeanWarps) sh.mass[threadIdx.x] = sh.acc[0][threadIdx.x];
+                if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[0][threadIdx.x];
                 __syncthreads();
                 auto wf = [&](int vi, float(&w)[8]) {
                     float fp[8], fq[8];
@@ -453,7 +599,7 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
                         w[i] = fmaxf(t, 0.f);
                     }
                 };
-                tok = block_sample<8>(g, wf, sh.mass, ures, &sh.tok);
+                tok = block_sample2(g, wf, sh.mass, ures, &sh.tok);
             }
             if (tok < 0) {
                 o.status |= SPECHUB_ST_ZERO_RESIDUAL;
@@ -469,7 +615,8 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_verify_kernel(RowArgs a)
 // ------------------------------------------------------------------------------------------------
 // Draft step.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kLeanThreads, 2) lean_draft_kernel(RowArgs a, int method) {
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(RowArgs a, int method) {
     __shared__ LeanShared sh;
     const long long r = blockIdx.x;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
@@ -483,7 +630,8 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_draft_kernel(RowArgs a, 
 
     LeanAcc tq, unused;
     lean_pass_a<false>(vq, vq, lo, hi, lane, k, tq, unused);
-    const ArgMaxSum q = lean_reduce(tq, vq, lo, hi, k, 1, sh);
+    ArgMaxSum q, unusedq;
+    lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
     const float Zq = q.sx + 1.f;
     uint32_t st = 0;
     int x1 = -1, x2 = -1, hubtok = -1;
@@ -492,7 +640,7 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_draft_kernel(RowArgs a, 
         st = SPECHUB_ST_NONFINITE;
     } else {
         hubtok = q.idx;
-        x1 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u1, 1, sh);
+        x1 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u1, 0, sh);
         if (method == kSpecHub) {
             prob0 = 1.f / Zq;
             if (x1 != hubtok) {
@@ -502,13 +650,13 @@ __global__ void __launch_bounds__(kLeanThreads, 2) lean_draft_kernel(RowArgs a, 
                 x2 = (hubtok == 0) ? 1 : 0;
                 st |= SPECHUB_ST_DEGENERATE_Q;
             } else {
-                x2 = lean_sample_row(g, rowq, k, q.c, hubtok, hubtok, u2, 1, sh);
+                x2 = lean_sample_row(g, rowq, k, q.c, hubtok, hubtok, u2, 0, sh);
                 prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2), k, -q.c)) / q.sx;
             }
         } else if (method == kRRS) {
-            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u2, 1, sh);
+            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u2, 0, sh);
         } else {
-            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, x1, u2, 1, sh);
+            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, x1, u2, 0, sh);
             if (x2 < 0) {
                 x2 = (x1 == 0) ? 1 : 0;
                 st |= SPECHUB_ST_DEGENERATE_Q;
