@@ -34,6 +34,9 @@ struct LeanShared {
     int cand[2];                    // lowest index attaining the row maximum
     float acc[4][kLeanMaxWarps];
     float mass[kLeanMaxWarps];
+    float part[1024];  // sampler: per-thread block sums of the selected warp range
+    float tt2;
+    int blk;
     int tok;
 };
 
@@ -207,22 +210,24 @@ __device__ void lean_reduce2(const LeanAcc &tp, const LeanAcc &tq, const uint4 *
     Q.ml = rmq; Q.c = Cq; Q.idx = idxq; Q.sx = t1;
 }
 
-// CTA-wide inverse-CDF draw with two rounds of warp-parallel loads.  mass[w] (shared) = total
-// weight of warp w's range; weights(vi, w[8]) the weights of vector vi.  In the selected warp,
-// round 1 gives every lane a contiguous block of the range (one scan finds the block), round 2
-// spreads that block's vectors over the lanes (one scan finds the vector).  Same result rule as
-// block_sample.  Must be called by all threads of the CTA.
+// CTA-wide inverse-CDF draw.  mass[w] (shared) = total weight of warp w's range (the coarse CDF
+// from pass B); weights(vi, w[8]) the weights of vector vi.  Every thread knows the selected warp
+// range; round 1 cuts it into one contiguous block of vectors per thread of the CTA and sums the
+// blocks in parallel, warp 0 scans the block sums; round 2 spreads the chosen block's vectors over
+// the lanes of warp 0.  Two load round trips in all.  Returns to every thread the lowest id whose
+// inclusive prefix exceeds u * total; when rounding leaves none inside the selected range, the
+// last id with positive weight there; -1 when the total is 0.  Called by all threads of the CTA.
 template <class WF>
-__device__ int block_sample2(const Geo &g, WF weights, const float *mass, float u, int *sh_tok) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+__device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float u) {
+    const int lane = threadIdx.x & 31, nth = blockDim.x;
     float total = 0.f;
-    for (int w = 0; w < g.nwarps; ++w) total += mass[w];
+    for (int w = 0; w < g.nwarps; ++w) total += sh.mass[w];
     if (!(total > 0.f)) return -1;
     const float t = u * total;
     int wsel = -1, lastw = -1;
     float base = 0.f, lastbase = 0.f, run = 0.f;
     for (int w = 0; w < g.nwarps; ++w) {
-        const float m = mass[w];
+        const float m = sh.mass[w];
         if (m > 0.f) {
             lastw = w;
             lastbase = run;
@@ -231,12 +236,10 @@ __device__ int block_sample2(const Geo &g, WF weights, const float *mass, float 
         run += m;
     }
     if (wsel < 0) { wsel = lastw; base = lastbase; }
-    if (warp == wsel) {
-        const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
-        const int J = (hi - lo + 31) / 32;  // vectors per lane block
-        float tt = t - base;
-        // round 1: lane totals over contiguous blocks
-        const int b0 = lo + lane * J, b1 = min(hi, b0 + J);
+    const int lo = g.seg_lo(wsel), hi = g.seg_hi(wsel);
+    const int Bv = (hi - lo + nth - 1) / nth;  // vectors per thread block
+    {   // round 1
+        const int b0 = lo + threadIdx.x * Bv, b1 = min(hi, b0 + Bv);
         float tot = 0.f;
 #pragma unroll 4
         for (int vi = b0; vi < b1; ++vi) {
@@ -244,20 +247,52 @@ __device__ int block_sample2(const Geo &g, WF weights, const float *mass, float 
             weights(vi, w);
             tot += ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
         }
-        float incl = tot;
+        sh.part[threadIdx.x] = tot;
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const float tt = t - base;
+        const int per = nth >> 5;  // block sums per lane
+        float ls = 0.f;
+        for (int i = 0; i < per; ++i) ls += sh.part[lane * per + i];
+        float incl = ls;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float up = __shfl_up_sync(kFull, incl, o);
             if (lane >= o) incl += up;
         }
-        const unsigned pos = __ballot_sync(kFull, tot > 0.f);
-        const unsigned hit = __ballot_sync(kFull, tot > 0.f && incl > tt);
-        int found = -1;
+        const unsigned pos = __ballot_sync(kFull, ls > 0.f);
+        const unsigned hit = __ballot_sync(kFull, ls > 0.f && incl > tt);
+        int blk = -1;
+        float tt2 = 0.f;
         if (pos) {
             const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
-            tt -= __shfl_sync(kFull, incl - tot, L);
-            const int c0 = lo + L * J, c1 = min(hi, c0 + J);
-            // round 2: the block's vectors over the lanes
+            if (lane == L) {
+                float acc = incl - ls;
+                int lastb = -1;
+                float lastacc = 0.f;
+                for (int i = 0; i < per; ++i) {
+                    const float m = sh.part[lane * per + i];
+                    if (m > 0.f) {
+                        lastb = lane * per + i;
+                        lastacc = acc;
+                        if (blk < 0 && acc + m > tt) { blk = lastb; tt2 = tt - acc; }
+                    }
+                    acc += m;
+                }
+                if (blk < 0) { blk = lastb; tt2 = tt - lastacc; }
+                sh.blk = blk;
+                sh.tt2 = tt2;
+            }
+        } else if (lane == 0) {
+            sh.blk = -1;
+        }
+        __syncwarp();
+        blk = sh.blk;
+        tt2 = sh.tt2;
+        int found = -1;
+        if (blk >= 0) {   // round 2: the block's vectors over the lanes
+            const int c0 = lo + blk * Bv, c1 = min(hi, c0 + Bv);
             float prefix = 0.f;
             int lastpos = -1;
             for (int v0 = c0; v0 < c1 && found < 0; v0 += 32) {
@@ -283,7 +318,7 @@ __device__ int block_sample2(const Geo &g, WF weights, const float *mass, float 
                     if (lane >= o) in2 += up;
                 }
                 const float tot2 = __shfl_sync(kFull, in2, 31);
-                const unsigned hit2 = __ballot_sync(kFull, lsum > 0.f && prefix + in2 > tt);
+                const unsigned hit2 = __ballot_sync(kFull, lsum > 0.f && prefix + in2 > tt2);
                 if (hit2) {
                     const int M = __ffs(hit2) - 1;
                     int cand = -1;
@@ -295,7 +330,7 @@ __device__ int block_sample2(const Geo &g, WF weights, const float *mass, float 
                             acc += w[i];
                             if (w[i] > 0.f) {
                                 lastin = vi * 8 + i;
-                                if (cand < 0 && acc > tt) cand = lastin;
+                                if (cand < 0 && acc > tt2) cand = lastin;
                             }
                         }
                         if (cand < 0) cand = lastin;
@@ -310,10 +345,10 @@ __device__ int block_sample2(const Geo &g, WF weights, const float *mass, float 
             }
             if (found < 0) found = lastpos;
         }
-        if (lane == 0) *sh_tok = found;
+        if (lane == 0) sh.tok = found;
     }
     __syncthreads();
-    const int tok = *sh_tok;
+    const int tok = sh.tok;
     __syncthreads();
     return tok;
 }
@@ -350,7 +385,7 @@ __device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, 
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
     };
-    return block_sample2(g, wf, sh.mass, u, &sh.tok);
+    return block_sample3(g, wf, sh, u);
 }
 
 template <int NACC>
@@ -495,7 +530,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
                 }
             };
-            int tok = block_sample2(g, wf, sh.mass, ures, &sh.tok);
+            int tok = block_sample3(g, wf, sh, ures);
             if (tok < 0) {
                 o.status |= SPECHUB_ST_ZERO_RESIDUAL;
                 tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
@@ -599,7 +634,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                         w[i] = fmaxf(t, 0.f);
                     }
                 };
-                tok = block_sample2(g, wf, sh.mass, ures, &sh.tok);
+                tok = block_sample3(g, wf, sh, ures);
             }
             if (tok < 0) {
                 o.status |= SPECHUB_ST_ZERO_RESIDUAL;
