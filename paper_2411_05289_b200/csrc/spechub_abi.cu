@@ -63,12 +63,47 @@ RowArgs base_args(const spechub_desc *d) {
 
 // The lean kernels take bf16 rows whose starts are 16-byte aligned and whose length is a
 // multiple of 8 and large enough to keep 512 threads busy.
-int lean_threads(const spechub_desc *d) {
+constexpr int kLeanThreads = 256;  // 4 CTAs per SM measured best (256/512/1024: 1.54/1.65/1.87 ms)
+
+// CTAs per row.  A row is split when its (target, draft) pair is large: with 4 CTAs per SM and
+// 148 SMs, 592/CS rows are between their first and second read at any time, and that many row
+// pairs should fit in L2 (126 MB) with room to spare.
+int lean_split(const spechub_desc *d) {
 #ifdef SPECHUB_TUNE
-    if (getenv("SPECHUB_T")) return atoi(getenv("SPECHUB_T"));
+    if (getenv("SPECHUB_CS")) return atoi(getenv("SPECHUB_CS"));
 #endif
-    (void)d;
-    return 256;  // 4 CTAs (rows) per SM measured best: 1.54 ms vs 1.65 (512) and 1.87 (1024) on V = 128256
+    const long long pair_bytes = 4LL * d->vocab;
+    if (pair_bytes * 592 <= (48LL << 20)) return 1;
+    if (pair_bytes * 296 <= (48LL << 20)) return 2;
+    return 4;
+}
+
+template <class K, class... Args>
+int launch_group(K kern, int cs, unsigned rows, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = cs > 1 ? 1 : 0;
+    cfg.gridDim = dim3(rows * cs); cfg.blockDim = dim3(kLeanThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+    return cudaLaunchKernelEx(&cfg, kern, args...) == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+}
+
+template <int CS>
+int launch_lean_verify_cs(int method, const RowArgs &a, unsigned rows, cudaStream_t s) {
+    if (method == kSpecHub) return launch_group(lean_verify_kernel<kSpecHub, kLeanThreads, CS>, CS, rows, s, a);
+    if (method == kRRS) return launch_group(lean_verify_kernel<kRRS, kLeanThreads, CS>, CS, rows, s, a);
+    return launch_group(lean_verify_kernel<kRRSw, kLeanThreads, CS>, CS, rows, s, a);
+}
+int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
+    if (cs == 4) return launch_lean_verify_cs<4>(method, a, rows, s);
+    if (cs == 2) return launch_lean_verify_cs<2>(method, a, rows, s);
+    return launch_lean_verify_cs<1>(method, a, rows, s);
+}
+int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
+    if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
+    if (cs == 2) return launch_group(lean_draft_kernel<kLeanThreads, 2>, 2, rows, s, a, method);
+    return launch_group(lean_draft_kernel<kLeanThreads, 1>, 1, rows, s, a, method);
 }
 
 bool lean_ok(const spechub_desc *d, bool aligned) {
@@ -96,10 +131,8 @@ int draft_common(const spechub_desc *d, const void *draft_logits, const float *u
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, draft_logits);
     if (lean_ok(d, al)) {
-        const int lt = lean_threads(d);
-        if (lt == 1024) lean_draft_kernel<1024><<<rows, 1024, 0, s>>>(a, method);
-        else if (lt == 512) lean_draft_kernel<512><<<rows, 512, 0, s>>>(a, method);
-        else lean_draft_kernel<256><<<rows, 256, 0, s>>>(a, method);
+        const int lrc = launch_lean_draft(method, lean_split(d), a, rows, s);
+        if (lrc != SPECHUB_OK) return lrc;
     } else if (d->dtype == SPECHUB_BF16) {
         if (al) draft_rows_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(a, method);
         else draft_rows_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(a, method);
@@ -150,20 +183,8 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, target_logits) && rows_aligned(d, draft_logits);
     if (lean_ok(d, al)) {
-        const int lt = lean_threads(d);
-        if (lt == 1024) {
-            if (method == kSpecHub) lean_verify_kernel<kSpecHub, 1024><<<rows, 1024, 0, s>>>(a);
-            else if (method == kRRS) lean_verify_kernel<kRRS, 1024><<<rows, 1024, 0, s>>>(a);
-            else lean_verify_kernel<kRRSw, 1024><<<rows, 1024, 0, s>>>(a);
-        } else if (lt == 512) {
-            if (method == kSpecHub) lean_verify_kernel<kSpecHub, 512><<<rows, 512, 0, s>>>(a);
-            else if (method == kRRS) lean_verify_kernel<kRRS, 512><<<rows, 512, 0, s>>>(a);
-            else lean_verify_kernel<kRRSw, 512><<<rows, 512, 0, s>>>(a);
-        } else {
-            if (method == kSpecHub) lean_verify_kernel<kSpecHub, 256><<<rows, 256, 0, s>>>(a);
-            else if (method == kRRS) lean_verify_kernel<kRRS, 256><<<rows, 256, 0, s>>>(a);
-            else lean_verify_kernel<kRRSw, 256><<<rows, 256, 0, s>>>(a);
-        }
+        const int lrc = launch_lean_verify(method, lean_split(d), a, rows, s);
+        if (lrc != SPECHUB_OK) return lrc;
     } else if (method == kSpecHub) launch_verify<kSpecHub>(d, a, al, rows, th, s);
     else if (method == kRRS) launch_verify<kRRS>(d, a, al, rows, th, s);
     else launch_verify<kRRSw>(d, a, al, rows, th, s);

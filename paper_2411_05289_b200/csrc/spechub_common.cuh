@@ -99,17 +99,24 @@ __device__ __forceinline__ float load_one<__nv_bfloat16>(const __nv_bfloat16 *ro
 }
 
 // How a row is cut over the warps of a CTA.
+// v0 / nloc describe the part of the row this CTA works on (the whole row unless the row is split
+// over the CTAs of a cluster); vector indices are always absolute.
 struct Geo {
-    int V, nvec, seg, nwarps;
-    __device__ __forceinline__ int seg_lo(int w) const { return min(w * seg, nvec); }
-    __device__ __forceinline__ int seg_hi(int w) const { return min((w + 1) * seg, nvec); }
+    int V, nvec, seg, nwarps, v0, nloc;
+    __device__ __forceinline__ int seg_lo(int w) const { return v0 + min(w * seg, nloc); }
+    __device__ __forceinline__ int seg_hi(int w) const { return v0 + min((w + 1) * seg, nloc); }
+    __device__ __forceinline__ bool holds_vec(int vi) const { return vi >= v0 && vi < v0 + nloc; }
+    __device__ __forceinline__ int warp_of_vec(int vi) const { return (vi - v0) / seg; }
 };
-__device__ __forceinline__ Geo make_geo(int V, int VW) {
+__device__ __forceinline__ Geo make_geo(int V, int VW, int parts = 1, int part = 0) {
     Geo g;
     g.V = V;
     g.nvec = (V + VW - 1) / VW;
     g.nwarps = blockDim.x >> 5;
-    g.seg = (g.nvec + g.nwarps - 1) / g.nwarps;
+    const int per = (g.nvec + parts - 1) / parts;
+    g.v0 = min(part * per, g.nvec);
+    g.nloc = min(per, g.nvec - g.v0);
+    g.seg = max(1, (g.nloc + g.nwarps - 1) / g.nwarps);
     return g;
 }
 

@@ -1,8 +1,15 @@
 // Lean streaming kernels for bf16 rows with 16-byte aligned starts and V % 8 == 0
-// (the shapes of the large-vocabulary workloads).  One CTA per (sequence, node)
-// row, several CTAs per SM so that one row's reductions overlap another row's
-// streaming.  Compared with the general kernels in spechub_stream.cuh the inner
-// loops are branch-free and carry no index bookkeeping:
+// (the shapes of the large-vocabulary workloads).  A (sequence, node) row is
+// worked on by a cluster of CS CTAs (CS = 1, 2 or 4), each owning a contiguous
+// slice of the vocabulary; several CTAs of different rows share an SM so that one
+// row's reductions overlap another row's streaming.  Splitting a row keeps the
+// number of rows in flight -- and with it the bytes between a row's first and
+// second read -- small enough that pass B hits L2 instead of HBM, without giving
+// up the thread count that hides latency.  The CTAs of a row meet at two or three
+// hardware cluster barriers and read each other's few partial results through
+// distributed shared memory.  Compared with the general kernels in
+// spechub_stream.cuh the inner loops are branch-free and carry no index
+// bookkeeping:
 //
 //   pass A  per 16-byte vector: a packed bf16 max tree (4 ops), 8 x (unpack, FMA,
 //           ex2, add).  The exponent reference c of a thread is the maximum of the
@@ -19,11 +26,14 @@
 // vocabulary pair per row.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "spechub.h"
 #include "spechub_common.cuh"
 #include "spechub_stream.cuh"
 
 namespace spechub {
+namespace cg = cooperative_groups;
 
 constexpr int kLeanMaxWarps = 32;
 constexpr float kHuge = 1.0e30f;  // ~2^100: partial sums beyond this move the reference
@@ -38,6 +48,30 @@ struct LeanShared {
     float tt2;
     int blk;
     int tok;
+    // what this CTA tells the other CTAs of its row (read through distributed shared memory)
+    float x_ml[2], x_sx[2];  // slice (max logit, sum without the slice argmax), 0 target / 1 draft
+    int x_idx[2];            // slice argmax
+    float x_sum[4];          // pass-B / pass-C sums of the slice
+    float x_mass;            // slice mass for a draw from q without a given token
+    int x_tok;               // a token drawn by this CTA
+};
+
+// The CTAs of one row.  CS = 1 compiles to no cluster instruction at all.
+template <int CS>
+struct RowGroup {
+    __device__ __forceinline__ static int rank() {
+        if (CS == 1) return 0;
+        return static_cast<int>(cg::this_cluster().block_rank());
+    }
+    __device__ __forceinline__ static void sync() {
+        if (CS == 1) __syncthreads();
+        else cg::this_cluster().sync();
+    }
+    template <class T>
+    __device__ __forceinline__ static const T *peer(const T *local, int r) {
+        if (CS == 1) return local;
+        return cg::this_cluster().map_shared_rank(local, r);
+    }
 };
 
 __device__ __forceinline__ unsigned bf2max(unsigned a, unsigned b) {
@@ -210,20 +244,17 @@ __device__ void lean_reduce2(const LeanAcc &tp, const LeanAcc &tq, const uint4 *
     Q.ml = rmq; Q.c = Cq; Q.idx = idxq; Q.sx = t1;
 }
 
-// CTA-wide inverse-CDF draw.  mass[w] (shared) = total weight of warp w's range (the coarse CDF
-// from pass B); weights(vi, w[8]) the weights of vector vi.  Every thread knows the selected warp
-// range; round 1 cuts it into one contiguous block of vectors per thread of the CTA and sums the
-// blocks in parallel, warp 0 scans the block sums; round 2 spreads the chosen block's vectors over
-// the lanes of warp 0.  Two load round trips in all.  Returns to every thread the lowest id whose
-// inclusive prefix exceeds u * total; when rounding leaves none inside the selected range, the
-// last id with positive weight there; -1 when the total is 0.  Called by all threads of the CTA.
+// CTA-wide inverse-CDF draw over this CTA's part of a row.  sh.mass[w] = total weight of warp w's
+// range (the coarse CDF); weights(vi, w[8]) the weights of vector vi; t = target prefix within
+// this part.  Every thread knows the selected warp range; round 1 cuts it into one contiguous
+// block of vectors per thread of the CTA and sums the blocks in parallel, warp 0 scans the block
+// sums; round 2 spreads the chosen block's vectors over the lanes of warp 0.  Two load round trips
+// in all.  Returns to every thread the lowest id whose inclusive prefix exceeds t; when rounding
+// leaves none inside the selected range, the last id with positive weight there; -1 when this
+// part has no mass.  Called by all threads of the CTA.
 template <class WF>
-__device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float u) {
+__device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) {
     const int lane = threadIdx.x & 31, nth = blockDim.x;
-    float total = 0.f;
-    for (int w = 0; w < g.nwarps; ++w) total += sh.mass[w];
-    if (!(total > 0.f)) return -1;
-    const float t = u * total;
     int wsel = -1, lastw = -1;
     float base = 0.f, lastbase = 0.f, run = 0.f;
     for (int w = 0; w < g.nwarps; ++w) {
@@ -235,6 +266,7 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float u) 
         }
         run += m;
     }
+    if (lastw < 0) return -1;
     if (wsel < 0) { wsel = lastw; base = lastbase; }
     const int lo = g.seg_lo(wsel), hi = g.seg_hi(wsel);
     const int Bv = (hi - lo + nth - 1) / nth;  // vectors per thread block
@@ -353,19 +385,77 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float u) 
     return tok;
 }
 
-// Draw from softmax(row), with token `excl` removed (excl < 0: none).  `hubtok` is the row's
-// argmax, whose exponential sh.wmass leaves out.
-__device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, float C, int hubtok,
-                               int excl, float u, int r, LeanShared &sh) {
+// Pick the CTA of a row whose part holds the target t of an inverse-CDF draw over per-CTA masses
+// m[0..n) (ascending token ranges).  Returns the rank (-1 if no mass) and the mass before it.
+__device__ __forceinline__ int pick_part(const float *m, int n, float t, float &base) {
+    int sel = -1, last = -1;
+    float lastbase = 0.f, run = 0.f;
+    base = 0.f;
+    for (int r = 0; r < n; ++r) {
+        if (m[r] > 0.f) {
+            last = r;
+            lastbase = run;
+            if (sel < 0 && run + m[r] > t) { sel = r; base = run; }
+        }
+        run += m[r];
+    }
+    if (sel < 0) { sel = last; base = lastbase; }
+    return sel;
+}
+
+// What every CTA of a row knows about one of its rows after the slices were merged.
+struct RowStat {
+    float ml, C, sx;  // row max logit, its shift, sum without the row argmax
+    int idx;          // row argmax
+};
+
+// Merge the slices' (max, argmax, sum without argmax) in rank order (Section 4: a = argmax q).
+template <int CS>
+__device__ __forceinline__ void merge_slices(const LeanShared &sh, int r, float k, RowStat &st) {
+    ArgMaxSum tot;
+    tot.init();
+#pragma unroll
+    for (int c = 0; c < CS; ++c) {
+        const LeanShared *ps = RowGroup<CS>::peer(&sh, c);
+        ArgMaxSum o;
+        o.ml = ps->x_ml[r]; o.c = shift_of(o.ml, k); o.sx = ps->x_sx[r]; o.idx = ps->x_idx[r];
+        tot = argmaxsum_merge(tot, o);
+    }
+    st.ml = tot.ml; st.C = tot.c; st.sx = tot.sx; st.idx = tot.idx;
+}
+
+// Mass of slice c of a row (row scale) for a draw from softmax(row) without token `excl`
+// (excl < 0: none; only a slice's own argmax can be left out here).  The slices' published
+// partials stay valid until the kernel ends.
+template <int CS>
+__device__ __forceinline__ float slice_mass(const LeanShared &sh, int r, const RowStat &st, int c, int excl,
+                                            float k) {
+    const LeanShared *ps = RowGroup<CS>::peer(&sh, c);
+    const float ml = ps->x_ml[r];
+    const float own = (ml > neg_inf() && ps->x_idx[r] != excl) ? 1.f : 0.f;
+    return (ps->x_sx[r] + own) * rescale(ml, shift_of(ml, k), st.C);
+}
+
+// Draw inside this CTA's slice from softmax(row) without token `excl`, target t (row scale,
+// relative to the start of the slice).  sh.wmass[r] holds the per-warp sums of the slice on the
+// slice's own scale with the slice argmax left out.
+__device__ int lean_sample_slice(const Geo &g, const __nv_bfloat16 *row, float k, const RowStat &st,
+                                 int excl, float t, int r, LeanShared &sh) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int locarg = sh.x_idx[r];
+    const float lml = sh.x_ml[r];
+    const float f = rescale(lml, shift_of(lml, k), st.C);
+    const float C = st.C;
     if (threadIdx.x < g.nwarps) {
         const int w = threadIdx.x;
-        const bool holds_hub = (hubtok / 8) >= g.seg_lo(w) && (hubtok / 8) < g.seg_hi(w);
-        sh.mass[w] = sh.wmass[r][w] + ((holds_hub && excl != hubtok) ? 1.f : 0.f);
+        const int lv = locarg >> 3;
+        const bool holds = lml > neg_inf() && lv >= g.seg_lo(w) && lv < g.seg_hi(w);
+        sh.mass[w] = (sh.wmass[r][w] + ((holds && excl != locarg) ? 1.f : 0.f)) * f;
     }
     __syncthreads();
-    if (excl >= 0 && excl != hubtok) {
-        const int wex = (excl / 8) / g.seg;
+    if (excl >= 0 && excl != locarg && g.holds_vec(excl >> 3)) {
+        // an arbitrary token of this slice is removed: its warp re-sums its range
+        const int wex = g.warp_of_vec(excl >> 3);
         if (warp == wex) {
             float s = 0.f;
             for (int vi = g.seg_lo(warp) + lane; vi < g.seg_hi(warp); vi += 32) {
@@ -385,7 +475,24 @@ __device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, 
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
     };
-    return block_sample3(g, wf, sh, u);
+    return block_sample3(g, wf, sh, t);
+}
+
+// Draw from softmax(row) without `excl` (the row argmax, a slice argmax, or nothing) over the
+// whole row: every CTA of the row calls it; the CTA whose slice holds the target draws and
+// returns the token, the others return -2.  -1: no mass.
+template <int CS>
+__device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, const RowStat &st, int me,
+                               int excl, float u, int r, LeanShared &sh) {
+    float m[CS];
+    float total = 0.f;
+#pragma unroll
+    for (int c = 0; c < CS; ++c) { m[c] = slice_mass<CS>(sh, r, st, c, excl, k); total += m[c]; }
+    if (!(total > 0.f)) return -1;
+    float base;
+    const int sel = pick_part(m, CS, u * total, base);
+    if (sel != me) return -2;
+    return lean_sample_slice(g, row, k, st, excl, u * total - base, r, sh);
 }
 
 template <int NACC>
@@ -406,305 +513,427 @@ __device__ __forceinline__ void lean_block_sums(float (&x)[NACC], LeanShared &sh
     }
 }
 
+// Sum NACC per-thread accumulators over the whole row: CTA sums, then the slices in rank order.
+// part[i][c] receives slice c's sum of accumulator i; sh.acc[i][w] keeps this CTA's per-warp sums.
+// Contains one row-group barrier.  OFF: first exchange slot used (a second call in the same
+// kernel takes other slots, so no CTA overwrites what a slower one has not read yet).
+template <int CS, int NACC, int OFF>
+__device__ __forceinline__ void lean_row_sums(float (&x)[NACC], float (&part)[NACC][CS], LeanShared &sh) {
+    lean_block_sums<NACC>(x, sh);
+    if (CS == 1) {
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) part[i][0] = x[i];
+        __syncthreads();  // sh.acc may be rewritten by a later sum only after all have read it
+        return;
+    }
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) sh.x_sum[OFF + i] = x[i];
+    }
+    RowGroup<CS>::sync();
+#pragma unroll
+    for (int i = 0; i < NACC; ++i) {
+        float t = 0.f;
+#pragma unroll
+        for (int c = 0; c < CS; ++c) {
+            part[i][c] = RowGroup<CS>::peer(&sh, c)->x_sum[OFF + i];
+            t += part[i][c];
+        }
+        x[i] = t;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
-template <int METHOD, int THREADS>
+template <int METHOD, int THREADS, int CS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(RowArgs a) {
     __shared__ LeanShared sh;
-    const long long r = blockIdx.x;
+    const int me = RowGroup<CS>::rank();
+    const long long r = blockIdx.x / CS;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
     const __nv_bfloat16 *rowp = static_cast<const __nv_bfloat16 *>(a.target) + b * a.stride_seq + n * a.stride_node;
     const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
     const uint4 *vp = reinterpret_cast<const uint4 *>(rowp), *vq = reinterpret_cast<const uint4 *>(rowq);
-    const Geo g = make_geo(a.vocab, 8);
+    const Geo g = make_geo(a.vocab, 8, CS, me);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
     const float k = kLog2e / temperature_of(a, b);
     const float r1 = a.uniforms[r * 5 + 2], r2 = a.uniforms[r * 5 + 3], ures = a.uniforms[r * 5 + 4];
     const float pinf = -neg_inf();
     const bool leaf = a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF;
+    const bool writer = (me == 0 && threadIdx.x == 0);
 
     NodeResult o;
     o.accept_idx = -1; o.token = -1; o.hub = -1; o.status = 0;
     o.beta[0] = o.beta[1] = 0.f; o.rate[0] = o.rate[1] = o.rate[2] = 0.f;
+    // The token is written by the CTA that knows it: the row's first CTA for an accepted draft or
+    // a flagged row, the CTA that draws for a residual / leaf token.
+    bool token_elsewhere = false;
 
     LeanAcc tp, tq;
     if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
-    ArgMaxSum P, Q;
-    if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, P, Q);
-    else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, P, Q);
-    const float Zp = P.sx + 1.f;
-    if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
-        o.status = SPECHUB_ST_NONFINITE;
-        if (threadIdx.x == 0) write_node(a, r, o);
-        return;
+    {
+        ArgMaxSum Ps, Qs;
+        if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        if (threadIdx.x == 0) {
+            sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
+            sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+        }
     }
-    const float cP = P.c, invZp = 1.f / Zp;
-    if (leaf) {
-        o.token = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
-        o.rate[2] = 1.f;
-        if (threadIdx.x == 0) write_node(a, r, o);
-        return;
-    }
-    const float Zq = Q.sx + 1.f;
-    if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) {
-        o.status = SPECHUB_ST_NONFINITE;
-        if (threadIdx.x == 0) write_node(a, r, o);
-        return;
-    }
-    const float cQ = Q.c, invZq = 1.f / Zq;
+    RowGroup<CS>::sync();  // [1] slices published
+    RowStat P, Q;
+    merge_slices<CS>(sh, 0, k, P);
+    merge_slices<CS>(sh, 1, k, Q);
+    const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
+    const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
     const int x1 = a.draft_tokens_in[2 * r], x2 = a.draft_tokens_in[2 * r + 1];
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
     auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
+    auto draw_from_p = [&]() {  // every CTA of the row calls it
+        const int tok = lean_sample_row<CS>(g, rowp, k, P, me, -1, ures, 0, sh);
+        if (tok != -2 && threadIdx.x == 0) a.token[r] = tok;
+        token_elsewhere = true;
+    };
 
-    if (METHOD == kSpecHub) {
-        const int hubtok = Q.idx;
-        o.hub = hubtok;
-        const bool pair_xa = (x2 == hubtok && x1 != hubtok), pair_ax = (x1 == hubtok && x2 != hubtok);
-        const int x = pair_xa ? x1 : x2;
-        if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) {
-            o.status = SPECHUB_ST_TOKEN_RANGE;
-            if (threadIdx.x == 0) write_node(a, r, o);
-            return;
+    do {
+        if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) { o.status = SPECHUB_ST_NONFINITE; break; }
+        if (leaf) {
+            // bonus token after the last accepted draft (Figure 2): a draw from p
+            draw_from_p();
+            o.rate[2] = 1.f;
+            break;
         }
-        const bool degenerate = !(Q.sx > 0.f);
-        const float c = degenerate ? 0.f : 1.f / Q.sx;
-        const float qa = invZq, rest = Q.sx * invZq;
-        const int hubvec = hubtok >> 3, hubel = hubtok & 7;
-        // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
-        float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
+        if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) { o.status = SPECHUB_ST_NONFINITE; break; }
+        if (METHOD == kSpecHub) {
+            const int hubtok = Q.idx;
+            o.hub = hubtok;
+            const bool pair_xa = (x2 == hubtok && x1 != hubtok), pair_ax = (x1 == hubtok && x2 != hubtok);
+            const int x = pair_xa ? x1 : x2;
+            if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
+            const bool degenerate = !(Q.sx > 0.f);
+            const float c = degenerate ? 0.f : 1.f / Q.sx;
+            const float qa = invZq, rest = Q.sx * invZq;
+            const int hubvec = hubtok >> 3, hubel = hubtok & 7;
+            // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
+            float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
 #pragma unroll 2
-        for (int vi = lo + lane; vi < hi; vi += 32) {
-            float fp[8], fq[8];
-            unpack_bf16x8(vp[vi], fp);
-            unpack_bf16x8(vq[vi], fq);
-            if (vi == hubvec) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i == hubel) { fp[i] = neg_inf(); fq[i] = neg_inf(); }
-            }
-#pragma unroll
-            for (int i = 0; i < 8; i += 2) {
-                float d, t;
-                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
-                s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
-                transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), c, d, t);
-                s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
-            }
-        }
-        float acc[3] = {s1a + s1b, s2a + s2b, ra + rb};
-        lean_block_sums<3>(acc, sh);
-        const float S1 = acc[0], S2 = degenerate ? qa : acc[1], R = acc[2];
-        const float pa = prob_p(hubtok);
-        const float hub_left = fmaxf(pa - S2, 0.f);
-        o.rate[0] = fmaxf(rest - S1, 0.f) + fminf(pa, S2);
-        o.rate[1] = (degenerate ? 0.f : fmaxf(qa - S2, 0.f)) + fminf(hub_left, S1);
-        o.rate[2] = R;
-        if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
-        const float px = prob_p(x), qx = prob_q(x);
-        bool acc1, acc2;
-        if (pair_xa) {
-            acc1 = accept_test(r1, px, qx, o.beta[0], true, o.status);
-            if (acc1) { o.accept_idx = 0; o.token = x; }
-            acc2 = accept_test(r2, hub_left, S1, o.beta[1], !acc1, o.status);
-            if (!acc1 && acc2) { o.accept_idx = 1; o.token = hubtok; }
-        } else {
-            acc1 = accept_test(r1, fmaxf(__fsub_rn(px, qx), 0.f), c * qx, o.beta[0], true, o.status);
-            if (acc1) { o.accept_idx = 1; o.token = x; }
-            acc2 = accept_test(r2, pa, S2, o.beta[1], !acc1, o.status);
-            if (!acc1 && acc2) { o.accept_idx = 0; o.token = hubtok; }
-        }
-        if (!(acc1 || acc2)) {
-            if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
-            __syncthreads();
-            auto wf = [&](int vi, float(&w)[8]) {
+            for (int vi = lo + lane; vi < hi; vi += 32) {
                 float fp[8], fq[8];
                 unpack_bf16x8(vp[vi], fp);
                 unpack_bf16x8(vq[vi], fq);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    float d, t;
-                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
-                    w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
-                }
-            };
-            int tok = block_sample3(g, wf, sh, ures);
-            if (tok < 0) {
-                o.status |= SPECHUB_ST_ZERO_RESIDUAL;
-                tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
-            }
-            o.accept_idx = -1;
-            o.token = tok;
-        }
-    } else {
-        if (x1 < 0 || x1 >= a.vocab || x2 < 0 || x2 >= a.vocab) {
-            o.status = SPECHUB_ST_TOKEN_RANGE;
-            if (threadIdx.x == 0) write_node(a, r, o);
-            return;
-        }
-        // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
-        const int x1vec = x1 >> 3, x1el = x1 & 7;
-        float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
-#pragma unroll 2
-        for (int vi = lo + lane; vi < hi; vi += 32) {
-            float fp[8], fq[8];
-            unpack_bf16x8(vp[vi], fp);
-            unpack_bf16x8(vq[vi], fq);
-            float pp[8], qq[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
-#pragma unroll
-            for (int i = 0; i < 8; i += 2) {
-                a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
-                a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
-            }
-            if (METHOD == kRRSw) {
-                if (vi == x1vec) {
+                if (vi == hubvec) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if (i == x1el) qq[i] = 0.f;
+                        if (i == hubel) { fp[i] = neg_inf(); fq[i] = neg_inf(); }
                 }
-                dna += (qq[0] + qq[1]) + (qq[2] + qq[3]);
-                dnb += (qq[4] + qq[5]) + (qq[6] + qq[7]);
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) {
+                    float d, t;
+                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                    s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
+                    transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), c, d, t);
+                    s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
+                }
             }
-        }
-        float acc[2] = {a1a + a1b, dna + dnb};
-        lean_block_sums<2>(acc, sh);
-        release_sums();
-        const float A1 = acc[0], den = acc[1];
-        const bool q1_zero = (METHOD == kRRSw) && !(den > 0.f);
-        const float gq = (METHOD == kRRSw) ? (q1_zero ? 0.f : 1.f / den) : 1.f;
-        const float A1g = A1 * gq;
-        // pass C: mass of the residual after two rejections
-        float w2a = 0.f, w2b = 0.f;
-#pragma unroll 2
-        for (int vi = lo + lane; vi < hi; vi += 32) {
-            float fp[8], fq[8];
-            unpack_bf16x8(vp[vi], fp);
-            unpack_bf16x8(vq[vi], fq);
-            float sc[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sc[i] = A1g;
-            if (METHOD == kRRSw && vi == x1vec) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i == x1el) sc[i] = 0.f;
+            float acc[3] = {s1a + s1b, s2a + s2b, ra + rb};
+            float part[3][CS];
+            lean_row_sums<CS, 3, 0>(acc, part, sh);  // [2]
+            const float S1 = acc[0], S2 = degenerate ? qa : acc[1], R = acc[2];
+            const float pa = prob_p(hubtok);
+            const float hub_left = fmaxf(pa - S2, 0.f);
+            o.rate[0] = fmaxf(rest - S1, 0.f) + fminf(pa, S2);
+            o.rate[1] = (degenerate ? 0.f : fmaxf(qa - S2, 0.f)) + fminf(hub_left, S1);
+            o.rate[2] = R;
+            if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
+            const float px = prob_p(x), qx = prob_q(x);
+            bool acc1, acc2;
+            if (pair_xa) {
+                acc1 = accept_test(r1, px, qx, o.beta[0], true, o.status);
+                if (acc1) { o.accept_idx = 0; o.token = x; }
+                acc2 = accept_test(r2, hub_left, S1, o.beta[1], !acc1, o.status);
+                if (!acc1 && acc2) { o.accept_idx = 1; o.token = hubtok; }
+            } else {
+                acc1 = accept_test(r1, fmaxf(__fsub_rn(px, qx), 0.f), c * qx, o.beta[0], true, o.status);
+                if (acc1) { o.accept_idx = 1; o.token = x; }
+                acc2 = accept_test(r2, pa, S2, o.beta[1], !acc1, o.status);
+                if (!acc1 && acc2) { o.accept_idx = 0; o.token = hubtok; }
             }
+            if (!(acc1 || acc2)) {
+                o.accept_idx = -1;
+                float base = 0.f;
+                const int sel = (R > 0.f) ? pick_part(part[2], CS, ures * R, base) : -1;
+                if (sel < 0) {
+                    o.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                    draw_from_p();
+                } else {
+                    token_elsewhere = true;
+                    if (sel == me) {
+                        if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
+                        __syncthreads();
+                        auto wf = [&](int vi, float(&w)[8]) {
+                            float fp[8], fq[8];
+                            unpack_bf16x8(vp[vi], fp);
+                            unpack_bf16x8(vq[vi], fq);
 #pragma unroll
-            for (int i = 0; i < 8; i += 2) {
-                float d, t;
-                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc[i], d, t);
-                w2a += fmaxf(t, 0.f);
-                transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), sc[i + 1], d, t);
-                w2b += fmaxf(t, 0.f);
-            }
-        }
-        float w2[1] = {w2a + w2b};
-        lean_block_sums<1>(w2, sh);
-        const float W2 = w2[0];
-        o.rate[0] = fmaxf(1.f - A1, 0.f);
-        o.rate[1] = fmaxf(A1 - W2, 0.f);
-        o.rate[2] = W2;
-        const float px1 = prob_p(x1), qx1 = prob_q(x1), px2 = prob_p(x2), qx2 = prob_q(x2);
-        const bool acc1 = accept_test(r1, px1, qx1, o.beta[0], true, o.status);
-        if (acc1) { o.accept_idx = 0; o.token = x1; }
-        if (!acc1 && q1_zero) o.status |= SPECHUB_ST_DEGENERATE_Q;
-        bool acc2 = false;
-        if (A1 > 0.f) {
-            const float q1x2 = (METHOD == kRRSw && x2 == x1) ? 0.f : A1g * qx2;
-            acc2 = accept_test(r2, fmaxf(__fsub_rn(px2, qx2), 0.f), q1x2, o.beta[1], !acc1, o.status);
-        }
-        if (!acc1 && acc2) { o.accept_idx = 1; o.token = x2; }
-        if (!(acc1 || acc2)) {
-            int tok = -1;
-            if (A1 > 0.f) {
-                if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[0][threadIdx.x];
-                __syncthreads();
-                auto wf = [&](int vi, float(&w)[8]) {
-                    float fp[8], fq[8];
-                    unpack_bf16x8(vp[vi], fp);
-                    unpack_bf16x8(vq[vi], fq);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float d, t;
-                        const float s = (METHOD == kRRSw && vi * 8 + i == x1) ? 0.f : A1g;
-                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), s, d, t);
-                        w[i] = fmaxf(t, 0.f);
+                            for (int i = 0; i < 8; ++i) {
+                                float d, t;
+                                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                                w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
+                            }
+                        };
+                        const int tok = block_sample3(g, wf, sh, ures * R - base);
+                        if (threadIdx.x == 0) a.token[r] = tok;
                     }
-                };
-                tok = block_sample3(g, wf, sh, ures);
+                }
             }
-            if (tok < 0) {
-                o.status |= SPECHUB_ST_ZERO_RESIDUAL;
-                tok = lean_sample_row(g, rowp, k, cP, P.idx, -1, ures, 0, sh);
+        } else {
+            if (x1 < 0 || x1 >= a.vocab || x2 < 0 || x2 >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
+            // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
+            const int x1vec = x1 >> 3, x1el = x1 & 7;
+            float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
+#pragma unroll 2
+            for (int vi = lo + lane; vi < hi; vi += 32) {
+                float fp[8], fq[8];
+                unpack_bf16x8(vp[vi], fp);
+                unpack_bf16x8(vq[vi], fq);
+                float pp[8], qq[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) {
+                    a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
+                    a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
+                }
+                if (METHOD == kRRSw) {
+                    if (vi == x1vec) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i == x1el) qq[i] = 0.f;
+                    }
+                    dna += (qq[0] + qq[1]) + (qq[2] + qq[3]);
+                    dnb += (qq[4] + qq[5]) + (qq[6] + qq[7]);
+                }
             }
-            o.accept_idx = -1;
-            o.token = tok;
+            float acc[2] = {a1a + a1b, dna + dnb};
+            float part2[2][CS];
+            lean_row_sums<CS, 2, 0>(acc, part2, sh);  // [2]
+            const float A1 = acc[0], den = acc[1];
+            const bool q1_zero = (METHOD == kRRSw) && !(den > 0.f);
+            const float gq = (METHOD == kRRSw) ? (q1_zero ? 0.f : 1.f / den) : 1.f;
+            const float A1g = A1 * gq;
+            // pass C: mass of the residual after two rejections
+            float w2a = 0.f, w2b = 0.f;
+#pragma unroll 2
+            for (int vi = lo + lane; vi < hi; vi += 32) {
+                float fp[8], fq[8];
+                unpack_bf16x8(vp[vi], fp);
+                unpack_bf16x8(vq[vi], fq);
+                float sc[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sc[i] = A1g;
+                if (METHOD == kRRSw && vi == x1vec) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i == x1el) sc[i] = 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) {
+                    float d, t;
+                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc[i], d, t);
+                    w2a += fmaxf(t, 0.f);
+                    transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), sc[i + 1], d, t);
+                    w2b += fmaxf(t, 0.f);
+                }
+            }
+            float w2[1] = {w2a + w2b};
+            float part1[1][CS];
+            lean_row_sums<CS, 1, 2>(w2, part1, sh);  // [3]
+            const float W2 = w2[0];
+            o.rate[0] = fmaxf(1.f - A1, 0.f);
+            o.rate[1] = fmaxf(A1 - W2, 0.f);
+            o.rate[2] = W2;
+            const float px1 = prob_p(x1), qx1 = prob_q(x1), px2 = prob_p(x2), qx2 = prob_q(x2);
+            const bool acc1 = accept_test(r1, px1, qx1, o.beta[0], true, o.status);
+            if (acc1) { o.accept_idx = 0; o.token = x1; }
+            if (!acc1 && q1_zero) o.status |= SPECHUB_ST_DEGENERATE_Q;
+            bool acc2 = false;
+            if (A1 > 0.f) {
+                const float q1x2 = (METHOD == kRRSw && x2 == x1) ? 0.f : A1g * qx2;
+                acc2 = accept_test(r2, fmaxf(__fsub_rn(px2, qx2), 0.f), q1x2, o.beta[1], !acc1, o.status);
+            }
+            if (!acc1 && acc2) { o.accept_idx = 1; o.token = x2; }
+            if (!(acc1 || acc2)) {
+                o.accept_idx = -1;
+                float base = 0.f;
+                const int sel = (A1 > 0.f && W2 > 0.f) ? pick_part(part1[0], CS, ures * W2, base) : -1;
+                if (sel < 0) {
+                    o.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                    draw_from_p();
+                } else {
+                    token_elsewhere = true;
+                    if (sel == me) {
+                        if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[0][threadIdx.x];
+                        __syncthreads();
+                        auto wf = [&](int vi, float(&w)[8]) {
+                            float fp[8], fq[8];
+                            unpack_bf16x8(vp[vi], fp);
+                            unpack_bf16x8(vq[vi], fq);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                float d, t;
+                                const float s = (METHOD == kRRSw && vi * 8 + i == x1) ? 0.f : A1g;
+                                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), s, d, t);
+                                w[i] = fmaxf(t, 0.f);
+                            }
+                        };
+                        const int tok = block_sample3(g, wf, sh, ures * W2 - base);
+                        if (threadIdx.x == 0) a.token[r] = tok;
+                    }
+                }
+            }
         }
+    } while (false);
+    if (writer) {
+        a.accept_idx[r] = o.accept_idx;
+        if (!token_elsewhere) a.token[r] = o.token;
+        if (a.hub) a.hub[r] = o.hub;
+        if (a.beta) { a.beta[2 * r] = o.beta[0]; a.beta[2 * r + 1] = o.beta[1]; }
+        if (a.rate) { a.rate[3 * r] = o.rate[0]; a.rate[3 * r + 1] = o.rate[1]; a.rate[3 * r + 2] = o.rate[2]; }
+        if (a.status) a.status[r] = o.status;
     }
-    if (threadIdx.x == 0) write_node(a, r, o);
+    if (CS > 1) RowGroup<CS>::sync();  // no CTA leaves while another may still read its shared memory
 }
 
 // ------------------------------------------------------------------------------------------------
-// Draft step.
+// Draft step (Section 4 / Algorithm 3 for SpecHub; Algorithm 1 for RRS, RRSw).
 // ------------------------------------------------------------------------------------------------
-template <int THREADS>
+template <int THREADS, int CS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(RowArgs a, int method) {
     __shared__ LeanShared sh;
-    const long long r = blockIdx.x;
+    const int me = RowGroup<CS>::rank();
+    const long long r = blockIdx.x / CS;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
     const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
     const uint4 *vq = reinterpret_cast<const uint4 *>(rowq);
-    const Geo g = make_geo(a.vocab, 8);
+    const Geo g = make_geo(a.vocab, 8, CS, me);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
     const float k = kLog2e / temperature_of(a, b);
     const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
+    const bool writer = (me == 0 && threadIdx.x == 0);
 
     LeanAcc tq, unused;
     lean_pass_a<false>(vq, vq, lo, hi, lane, k, tq, unused);
-    ArgMaxSum q, unusedq;
-    lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
-    const float Zq = q.sx + 1.f;
+    {
+        ArgMaxSum q, unusedq;
+        lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
+        if (threadIdx.x == 0) { sh.x_ml[0] = q.ml; sh.x_sx[0] = q.sx; sh.x_idx[0] = q.idx; sh.x_tok = -3; }
+    }
+    RowGroup<CS>::sync();  // [1]
+    RowStat Q;
+    merge_slices<CS>(sh, 0, k, Q);
+    const float Zq = Q.sx + 1.f;
     uint32_t st = 0;
-    int x1 = -1, x2 = -1, hubtok = -1;
-    float prob0 = 0.f, prob1 = 0.f;
-    if (!(q.ml > neg_inf()) || !finite_pos(Zq) || !(q.ml < -neg_inf())) {
-        st = SPECHUB_ST_NONFINITE;
+    const bool bad = !(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf());
+    const int hubtok = bad ? -1 : Q.idx;
+    if (bad) {
+        if (writer) {
+            a.draft_tokens_out[2 * r] = -1; a.draft_tokens_out[2 * r + 1] = -1;
+            if (a.hub) a.hub[r] = -1;
+            if (a.draft_prob) { a.draft_prob[2 * r] = 0.f; a.draft_prob[2 * r + 1] = 0.f; }
+            if (a.status) a.status[r] = SPECHUB_ST_NONFINITE;
+        }
     } else {
-        hubtok = q.idx;
-        x1 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u1, 0, sh);
+        // x1 ~ q.  The CTA whose slice holds the target draws it and tells the others.
+        const int t1 = lean_sample_row<CS>(g, rowq, k, Q, me, -1, u1, 0, sh);
+        int x1 = t1;
+        if (CS > 1) {
+            if (t1 != -2 && threadIdx.x == 0) sh.x_tok = t1;
+            RowGroup<CS>::sync();  // [2]
+            x1 = -1;
+#pragma unroll
+            for (int c = 0; c < CS; ++c) {
+                const int v = RowGroup<CS>::peer(&sh, c)->x_tok;
+                if (v != -3) x1 = v;
+            }
+        }
+        float prob0 = 0.f, prob1 = 0.f;
+        bool x2_elsewhere = false;  // x2 (and its probability) written by the CTA that draws it
+        int x2 = -1;
         if (method == kSpecHub) {
             prob0 = 1.f / Zq;
             if (x1 != hubtok) {
                 x2 = hubtok;
-                prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -q.c)) / Zq;
-            } else if (!(q.sx > 0.f)) {
+                prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)) / Zq;
+            } else if (!(Q.sx > 0.f)) {
                 x2 = (hubtok == 0) ? 1 : 0;
                 st |= SPECHUB_ST_DEGENERATE_Q;
             } else {
-                x2 = lean_sample_row(g, rowq, k, q.c, hubtok, hubtok, u2, 0, sh);
-                prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2), k, -q.c)) / q.sx;
+                const int t2 = lean_sample_row<CS>(g, rowq, k, Q, me, hubtok, u2, 0, sh);
+                x2_elsewhere = true;
+                if (t2 != -2 && threadIdx.x == 0) {
+                    a.draft_tokens_out[2 * r + 1] = t2;
+                    if (a.draft_prob)
+                        a.draft_prob[2 * r + 1] = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, t2), k, -Q.C)) / Q.sx;
+                }
             }
         } else if (method == kRRS) {
-            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, -1, u2, 0, sh);
+            const int t2 = lean_sample_row<CS>(g, rowq, k, Q, me, -1, u2, 0, sh);
+            x2_elsewhere = true;
+            if (t2 != -2 && threadIdx.x == 0) a.draft_tokens_out[2 * r + 1] = t2;
         } else {
-            x2 = lean_sample_row(g, rowq, k, q.c, hubtok, x1, u2, 0, sh);
-            if (x2 < 0) {
-                x2 = (x1 == 0) ? 1 : 0;
+            // q with q(x1) set to 0: the slice that holds x1 re-sums itself without it (unless x1
+            // is that slice's argmax, which its published sum already leaves out)
+            const int per = (g.nvec + CS - 1) / CS;
+            const int ox = min((x1 >> 3) / per, CS - 1);
+            const bool resum = RowGroup<CS>::peer(&sh, ox)->x_idx[0] != x1;
+            if (resum && me == ox) {
+                float s = 0.f;
+                for (int vi = lo + lane; vi < hi; vi += 32) {
+                    float v[8];
+                    unpack_bf16x8(vq[vi], v);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) s += (vi * 8 + i == x1) ? 0.f : ex2(__fmaf_rn(v[i], k, -Q.C));
+                }
+                float accs[1] = {s};
+                lean_block_sums<1>(accs, sh);
+                if (threadIdx.x == 0) sh.x_mass = accs[0];
+                __syncthreads();
+            }
+            if (CS > 1 && resum) RowGroup<CS>::sync();  // [3]
+            float m[CS];
+            float total = 0.f;
+#pragma unroll
+            for (int c = 0; c < CS; ++c) {
+                m[c] = (c == ox && resum) ? RowGroup<CS>::peer(&sh, c)->x_mass : slice_mass<CS>(sh, 0, Q, c, x1, k);
+                total += m[c];
+            }
+            x2_elsewhere = true;
+            float base = 0.f;
+            const int sel = (total > 0.f) ? pick_part(m, CS, u2 * total, base) : -1;
+            if (sel < 0) {
                 st |= SPECHUB_ST_DEGENERATE_Q;
+                if (writer) a.draft_tokens_out[2 * r + 1] = (x1 == 0) ? 1 : 0;
+            } else if (sel == me) {
+                const int t2 = lean_sample_slice(g, rowq, k, Q, x1, u2 * total - base, 0, sh);
+                if (threadIdx.x == 0) a.draft_tokens_out[2 * r + 1] = t2;
             }
         }
+        if (writer) {
+            a.draft_tokens_out[2 * r] = x1;
+            if (!x2_elsewhere) a.draft_tokens_out[2 * r + 1] = x2;
+            if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;
+            if (a.draft_prob) {
+                a.draft_prob[2 * r] = prob0;
+                if (!x2_elsewhere) a.draft_prob[2 * r + 1] = prob1;
+            }
+            if (a.status) a.status[r] = st;
+        }
     }
-    if (threadIdx.x == 0) {
-        a.draft_tokens_out[2 * r] = x1;
-        a.draft_tokens_out[2 * r + 1] = x2;
-        if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;
-        if (a.draft_prob) { a.draft_prob[2 * r] = prob0; a.draft_prob[2 * r + 1] = prob1; }
-        if (a.status) a.status[r] = st;
-    }
+    if (CS > 1) RowGroup<CS>::sync();
 }
 
 }  // namespace spechub
