@@ -57,7 +57,7 @@ extern "C" {
 #define SPECHUB_OK 0
 #define SPECHUB_ERR_NULL (-1)        /* a required pointer is NULL                        */
 #define SPECHUB_ERR_VERSION (-2)     /* struct_size / version do not match this library   */
-#define SPECHUB_ERR_SHAPE (-3)       /* batch < 0, nodes < 1, vocab < 2, k != 2, levels < 1 */
+#define SPECHUB_ERR_SHAPE (-3)       /* batch < 0, nodes < 1, vocab < 2, k != 2, levels < 1, bad flags */
 #define SPECHUB_ERR_DTYPE (-4)       /* dtype is not SPECHUB_F32 / SPECHUB_BF16            */
 #define SPECHUB_ERR_STRIDE (-5)      /* stride_node < vocab or stride_seq too small        */
 #define SPECHUB_ERR_TEMPERATURE (-6) /* temperature not a finite number > 0               */
@@ -76,6 +76,13 @@ extern "C" {
 #define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
 #define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
 #define SPECHUB_ST_INTERNAL 32u       /* a bounded wait for an on-chip copy expired: row output is -1 */
+
+/* descriptor flags: how many CTAs of a thread-block cluster share one row in the large-vocabulary
+ * bf16 kernels (a tuning hint; results do not depend on it beyond fp32 summation order).  At most
+ * one of the three may be set; none = the library chooses. */
+#define SPECHUB_FLAG_SPLIT_1 1u
+#define SPECHUB_FLAG_SPLIT_2 2u
+#define SPECHUB_FLAG_SPLIT_4 4u
 
 /* node kinds */
 #define SPECHUB_NODE_VERIFY 0 /* run the accept/reject tests on the node's two drafts         */
@@ -98,7 +105,7 @@ typedef struct spechub_desc {
     const int32_t *child;   /* device [nodes][2]: node reached by accepting draft i, < 0 = none;
                                NULL = complete binary tree in heap order, child i of n is 2n+1+i */
     const uint8_t *node_kind; /* device [nodes]: SPECHUB_NODE_*; NULL = every node verifies    */
-    uint32_t flags;       /* reserved, must be 0                                             */
+    uint32_t flags;       /* SPECHUB_FLAG_* bits; 0 = library defaults                        */
 } spechub_desc;
 
 /* Per-node outputs, each a device array [batch][nodes] (x trailing count).

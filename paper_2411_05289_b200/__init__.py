@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     load_library,
     rrs_draft_sample,
     rrs_verify_tree,
+    set_row_split,
     spechub_draft_sample,
     spechub_verify_tree,
     status_string,

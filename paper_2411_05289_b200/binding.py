@@ -120,6 +120,18 @@ def _check(code: int):
         raise SpecHubError(code, status_string(code))
 
 
+# tuning hint for the large-vocabulary bf16 kernels: CTAs of a cluster per row (0 = library default)
+_split = 0
+
+
+def set_row_split(ctas: int) -> None:
+    """Force 1, 2 or 4 CTAs per row in the large-vocabulary kernels (0 restores the default)."""
+    global _split
+    if ctas not in (0, 1, 2, 4):
+        raise ValueError("row split must be 0, 1, 2 or 4")
+    _split = ctas
+
+
 @dataclass
 class Tree:
     """Token tree in level order.  ``child``/``node_kind`` are device tensors or None
@@ -192,7 +204,7 @@ def _desc(logits: torch.Tensor, tree: Tree, temperature) -> tuple:
         if tree.node_kind.dtype != torch.uint8 or tuple(tree.node_kind.shape) != (N,):
             raise ValueError("node_kind must be a uint8 [nodes] tensor")
         d.node_kind = tree.node_kind.data_ptr()
-    d.flags = 0
+    d.flags = _split  # SPECHUB_FLAG_SPLIT_n has the value n
     return d, keep
 
 

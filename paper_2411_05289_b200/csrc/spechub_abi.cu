@@ -26,7 +26,8 @@ int check_desc(const spechub_desc *d) {
     if (d->nodes == 1 && d->batch > 1 && d->stride_seq < d->vocab) return SPECHUB_ERR_STRIDE;
     if (!d->temperature_per_seq && !(d->temperature > 0.f && isfinite(d->temperature)))
         return SPECHUB_ERR_TEMPERATURE;
-    if (d->flags != 0) return SPECHUB_ERR_SHAPE;
+    const uint32_t split = d->flags & 7u;
+    if ((d->flags & ~7u) != 0 || (split & (split - 1)) != 0) return SPECHUB_ERR_SHAPE;
     if ((int64_t)d->batch * d->nodes > 0x7fffffffLL) return SPECHUB_ERR_SHAPE;
     return SPECHUB_OK;
 }
@@ -65,17 +66,17 @@ RowArgs base_args(const spechub_desc *d) {
 // multiple of 8 and large enough to keep 512 threads busy.
 constexpr int kLeanThreads = 256;  // 4 CTAs per SM measured best (256/512/1024: 1.54/1.65/1.87 ms)
 
-// CTAs per row.  A row is split when its (target, draft) pair is large: with 4 CTAs per SM and
-// 148 SMs, 592/CS rows are between their first and second read at any time, and that many row
-// pairs should fit in L2 (126 MB) with room to spare.
+// CTAs per row.  With 4 CTAs per SM and 148 SMs, 592/CS rows are between their first and second
+// read at any time; at CS = 4 on V = 128256 that fits L2 (DRAM reads drop from 2.0x to 1.0x the
+// algorithmic bytes) but the per-CTA fixed work grows 4x, and the two cancel (1.6 vs 1.8 ms).
 int lean_split(const spechub_desc *d) {
 #ifdef SPECHUB_TUNE
     if (getenv("SPECHUB_CS")) return atoi(getenv("SPECHUB_CS"));
 #endif
-    const long long pair_bytes = 4LL * d->vocab;
-    if (pair_bytes * 592 <= (48LL << 20)) return 1;
-    if (pair_bytes * 296 <= (48LL << 20)) return 2;
-    return 4;
+    if (d->flags & SPECHUB_FLAG_SPLIT_1) return 1;
+    if (d->flags & SPECHUB_FLAG_SPLIT_2) return 2;
+    if (d->flags & SPECHUB_FLAG_SPLIT_4) return 4;
+    return 1;  // measured on B200: the per-CTA fixed work of a split row still outweighs the L2 hits
 }
 
 template <class K, class... Args>
@@ -256,7 +257,7 @@ const char *spechub_status_string(int code) {
         case SPECHUB_OK: return "ok";
         case SPECHUB_ERR_NULL: return "a required pointer is NULL";
         case SPECHUB_ERR_VERSION: return "descriptor struct_size/version mismatch";
-        case SPECHUB_ERR_SHAPE: return "bad shape: need batch >= 0, nodes >= 1, vocab >= 2, k == 2, levels >= 1, flags == 0";
+        case SPECHUB_ERR_SHAPE: return "bad shape: need batch >= 0, nodes >= 1, vocab >= 2, k == 2, levels >= 1, valid flags";
         case SPECHUB_ERR_DTYPE: return "dtype must be SPECHUB_F32 or SPECHUB_BF16";
         case SPECHUB_ERR_STRIDE: return "strides too small for the given shape";
         case SPECHUB_ERR_TEMPERATURE: return "temperature must be finite and > 0";

@@ -108,8 +108,9 @@ def test_small_shapes(sh, V, dtype):
     assert s.rows and s2.rows
 
 
+@pytest.mark.parametrize("split", [1, 2, 4])
 @pytest.mark.parametrize("V", [4096, 8192, 9000, 12344, 16384, 16392, 24000, 40000, 70000, 81920])
-def test_lean_shapes(sh, V):
+def test_lean_shapes(sh, V, split):
     """bf16, aligned, V % 8 == 0: shapes that take the lean bf16 kernels (V >= 8192) or, below that, the general ones
     with ragged warp ranges."""
     rng = np.random.default_rng(V + 3)
@@ -125,8 +126,12 @@ def test_lean_shapes(sh, V):
     lp, lq = workloads.round_to_storage(lp, "bf16"), workloads.round_to_storage(lq, "bf16")
     un = random_uniforms(rng, B, N)
     T = np.array([1.0, 0.6, 1.3, 0.8, 1.0], np.float32)
-    run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="lean-dense")
-    run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="lean-paper")
+    sh.set_row_split(split)
+    try:
+        run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="lean-dense-split%d" % split)
+        run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="lean-paper-split%d" % split)
+    finally:
+        sh.set_row_split(0)
 
 
 def test_peaked_rows_keep_precision(sh):
@@ -205,7 +210,7 @@ def test_argument_errors(sh):
     assert call(d) == 0
     for field, val, code in [("k", 3, -3), ("vocab", 1, -3), ("dtype", 7, -4), ("version", 9, -2),
                              ("stride_node", 8, -5), ("temperature", 0.0, -6), ("levels", 0, -3),
-                             ("flags", 1, -3)]:
+                             ("flags", 8, -3), ("flags", 3, -3)]:
         dd, _ = binding._desc(x, sh.Tree.heap(3), 1.0)
         setattr(dd, field, val)
         assert call(dd) == code, field
@@ -326,10 +331,15 @@ def test_config3_sampled(sh, variant):
     print("%s %r" % (cfg.name, s))
 
 
-def test_config4_sampled(sh):
+@pytest.mark.parametrize("split", [0, 4])
+def test_config4_sampled(sh, split):
     cfg = workloads.CONFIGS["c4"]
-    s = sampled_parity(sh, cfg, 64, layouts=(False, True))
-    print("c4 %r" % s)
+    sh.set_row_split(split)
+    try:
+        s = sampled_parity(sh, cfg, 64, layouts=(False, True))
+    finally:
+        sh.set_row_split(0)
+    print("c4 split=%d %r" % (split, s))
 
 
 def test_config5_sampled(sh):
