@@ -885,30 +885,19 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
             x2_elsewhere = true;
             if (t2 != -2 && threadIdx.x == 0) a.draft_tokens_out[2 * r + 1] = t2;
         } else {
-            // q with q(x1) set to 0: the slice that holds x1 re-sums itself without it (unless x1
-            // is that slice's argmax, which its published sum already leaves out)
+            // q with q(x1) set to 0.  The mass of the slice that holds x1 is its sum minus x1's term:
+            // unless x1 is that slice's argmax (which the published sum already leaves out), the
+            // argmax's own term stays in, so at most half of the sum cancels.
             const int per = (g.nvec + CS - 1) / CS;
             const int ox = min((x1 >> 3) / per, CS - 1);
-            const bool resum = RowGroup<CS>::peer(&sh, ox)->x_idx[0] != x1;
-            if (resum && me == ox) {
-                float s = 0.f;
-                for (int vi = lo + lane; vi < hi; vi += 32) {
-                    float v[8];
-                    unpack_bf16x8(vq[vi], v);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) s += (vi * 8 + i == x1) ? 0.f : ex2(__fmaf_rn(v[i], k, -Q.C));
-                }
-                float accs[1] = {s};
-                lean_block_sums<1>(accs, sh);
-                if (threadIdx.x == 0) sh.x_mass = accs[0];
-                __syncthreads();
-            }
-            if (CS > 1 && resum) RowGroup<CS>::sync();  // [3]
+            const float lx1 = load_one<__nv_bfloat16>(rowq, x1);
             float m[CS];
             float total = 0.f;
 #pragma unroll
             for (int c = 0; c < CS; ++c) {
-                m[c] = (c == ox && resum) ? RowGroup<CS>::peer(&sh, c)->x_mass : slice_mass<CS>(sh, 0, Q, c, x1, k);
+                m[c] = slice_mass<CS>(sh, 0, Q, c, x1, k);
+                if (c == ox && RowGroup<CS>::peer(&sh, c)->x_idx[0] != x1)
+                    m[c] = fmaxf(m[c] - ex2(__fmaf_rn(lx1, k, -Q.C)), 0.f);
                 total += m[c];
             }
             x2_elsewhere = true;
