@@ -33,6 +33,11 @@ METRIC = "tree-nodes verified/sec"
 UNIT = "nodes/s"
 METHODS = ("spechub", "rrs", "rrsw")
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+# profiles/, scaled from the captured batch to the workload's batch (traffic grows with the row
+# count).  Keyed by (API call, workload); absent = not captured for the current kernels.
+TRAFFIC = {}
+
 
 def parse():
     ap = argparse.ArgumentParser()
@@ -222,24 +227,31 @@ def main():
 
     outs = {m: alloc_verify_outputs(B, N, tree.levels, dev) for m in METHODS}
     stream = torch.cuda.current_stream()
-    ev_pairs = []
+    ev_pairs = {}  # API call -> list of (start, stop) events recorded inside the timed steps
+
+    def timed(name, record, fn):
+        if not record:
+            return fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        r = fn()
+        e1.record(stream)
+        ev_pairs.setdefault(name, []).append((e0, e1))
+        return r
 
     def step(record=False):
         for m in METHODS:
             if m == "spechub":
-                d = sh.spechub_draft_sample(tq, un, tree, cfg.temperature)
+                d = timed("spechub_draft_sample", record,
+                          lambda: sh.spechub_draft_sample(tq, un, tree, cfg.temperature))
+                timed("spechub_verify_tree", record,
+                      lambda: sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=outs[m]))
             else:
-                d = sh.rrs_draft_sample(tq, un, tree, m == "rrsw", cfg.temperature)
-            if record and m == "spechub":
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-            if m == "spechub":
-                sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=outs[m])
-            else:
-                sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=outs[m])
-            if record and m == "spechub":
-                e1.record(stream)
-                ev_pairs.append((e0, e1))
+                wo = m == "rrsw"
+                d = timed("rrs_draft_sample[%s]" % m, record,
+                          lambda: sh.rrs_draft_sample(tq, un, tree, wo, cfg.temperature))
+                timed("rrs_verify_tree[%s]" % m, record,
+                      lambda: sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, wo, cfg.temperature, out=outs[m]))
 
     def barrier():
         torch.cuda.synchronize()
@@ -268,8 +280,9 @@ def main():
     barrier()
     ms = t0.elapsed_time(t1)
     clocks = clk.stop() if rank == 0 else None
-    # the walk kernel is inside the recorded span; it is a few microseconds
-    verify_ms = float(np.mean([a.elapsed_time(b) for a, b in ev_pairs]))
+    # per API call: mean device time of its kernels (a verify call = verification kernel + walk kernel)
+    call_ms = {k: float(np.mean([a.elapsed_time(b) for a, b in v])) for k, v in ev_pairs.items()}
+    verify_ms = call_ms["spechub_verify_tree"]
 
     # ---- end to end: host buffers in, host results out, through the public API ----
     esz = 2 if cfg.dtype == "bf16" else 4
@@ -293,11 +306,13 @@ def main():
 
     e2e_step()
     barrier()
-    w0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(stream)
     for _ in range(args.e2e_steps):
         e2e_step()
+    g1.record(stream)
     barrier()
-    e2e_s = time.perf_counter() - w0
+    e2e_s = g0.elapsed_time(g1) * 1e-3
 
     tms = torch.tensor([ms, e2e_s * 1e3, verify_ms], device=dev, dtype=torch.float64)
     if world > 1:
@@ -311,8 +326,17 @@ def main():
         kind = workloads.paper_node_kind(N) if args.layout == "paper" else np.zeros(N, np.uint8)
         n_leaf = int(kind.sum())
         alg_bytes = B * ((N - n_leaf) * (2 * V * esz + 8 + 20 + 44) + n_leaf * (V * esz + 20 + 44))
+        draft_bytes = B * N * (V * esz + 8 + 8 + 16)
         peak, peak_src = measured_peak()
-        achieved = alg_bytes / (verify_ms * 1e-3) / 1e9
+        total_call_ms = sum(call_ms.values())
+        roof = {}
+        for name, t_ms in call_ms.items():
+            nbytes = draft_bytes if "draft" in name else alg_bytes
+            ach = nbytes / (t_ms * 1e-3) / 1e9
+            roof[name] = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
+                          "frac": ach / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0,
+                          "traffic": TRAFFIC.get((name, cfg.name)), "alg_bytes_per_launch": nbytes,
+                          "ms_per_launch": t_ms, "share_of_step": t_ms / total_call_ms}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -322,16 +346,23 @@ def main():
                     "steps": args.e2e_steps},
             "gpu_launches": 9 * args.steps,
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "spechub_verify_tree (verification kernel + walk)",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / 8000.0,
-                         "traffic": None, "alg_bytes_per_launch": alg_bytes, "ms_per_launch": verify_ms},
+            "roofline": roof["spechub_verify_tree"],
+            "kernels": roof,
+            "special_function_pipe": {
+                "note": "4 ex2 per vocabulary pair per verified row (2 in pass A, 2 in pass B); "
+                        "B200 issues 16 ex2/clk/SM (measured)",
+                "kernel": "spechub_verify_tree",
+                "achieved_ex2_per_s": 4.0 * B * (N - n_leaf) * V / (verify_ms * 1e-3),
+                "peak_ex2_per_s": 148 * 16 * (clocks["sm_mhz"] or 1965.0) * 1e6,
+            },
             "breakdown": {
                 "spechub_verify_nodes_per_s": B * N / (verify_ms * 1e-3),
                 "spechub_verify_vocab_elements_per_s": B * N * V / (verify_ms * 1e-3),
                 "step_vocab_elements_per_s": nodes_per_step * V * args.steps / (ms * 1e-3),
             },
         }
+        sfp = line["special_function_pipe"]
+        sfp["frac"] = sfp["achieved_ex2_per_s"] / sfp["peak_ex2_per_s"]
         if not args.no_cpu_baseline and world == 1:
             v, desc, _ = oracle_sample(cfg, args.layout, args.cpu_seconds)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
