@@ -558,6 +558,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     const Geo g = make_geo(a.vocab, 8, CS, me);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    // Pass B walks this lane's vectors backwards: what pass A read last is read again first, so
+    // the tail of the row is still in L2 even when the rows in flight exceed its capacity.
+    const int last_vi = (lo + lane < hi) ? lo + lane + ((hi - 1 - lo - lane) / 32) * 32 : lo - 1;
     const float k = kLog2e / temperature_of(a, b);
     const float r1 = a.uniforms[r * 5 + 2], r2 = a.uniforms[r * 5 + 3], ures = a.uniforms[r * 5 + 4];
     const float pinf = -neg_inf();
@@ -620,7 +623,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
             float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
 #pragma unroll 2
-            for (int vi = lo + lane; vi < hi; vi += 32) {
+            for (int vi = last_vi; vi >= lo; vi -= 32) {
                 float fp[8], fq[8];
                 unpack_bf16x8(vp[vi], fp);
                 unpack_bf16x8(vq[vi], fq);
@@ -695,7 +698,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             const int x1vec = x1 >> 3, x1el = x1 & 7;
             float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
 #pragma unroll 2
-            for (int vi = lo + lane; vi < hi; vi += 32) {
+            for (int vi = last_vi; vi >= lo; vi -= 32) {
                 float fp[8], fq[8];
                 unpack_bf16x8(vp[vi], fp);
                 unpack_bf16x8(vq[vi], fq);
