@@ -109,7 +109,9 @@ typedef struct spechub_desc {
 } spechub_desc;
 
 /* Per-node outputs, each a device array [batch][nodes] (x trailing count).
- * accept_idx and token are required; the others may be NULL. */
+ * accept_idx and token are required; the others may be NULL.  When beta and rate are both NULL
+ * no probability is reported, and a row whose first test accepts is finished after the first
+ * pass over its logits (the transport sums could not change its outcome). */
 typedef struct spechub_node_out {
     int32_t *accept_idx; /* 0 / 1: child whose draft was accepted; -1: rejected, leaf or flagged */
     int32_t *token;      /* token emitted at this node: accepted draft, residual or leaf draw;

@@ -267,7 +267,7 @@ def alloc_verify_outputs(B, N, levels, dev):
 
 
 def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream,
-            out):
+            out, probabilities=True):
     lib = load_library()
     _same_layout(target_logits, draft_logits)
     d, keep = _desc(target_logits, tree, temperature)
@@ -279,7 +279,8 @@ def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, t
         raise ValueError("draft_tokens must be a contiguous int32 [batch][nodes][2] tensor")
     if out is None:
         out = alloc_verify_outputs(B, N, tree.levels, dev)
-    no = _NodeOut(*[out[k].data_ptr() for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
+    no = _NodeOut(*[out[k].data_ptr() if (probabilities or k not in ("beta", "rate")) else None
+                    for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
     so = _SeqOut(*[out[k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])
     ws_bytes = lib.spechub_workspace_bytes(ctypes.byref(d))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
@@ -293,18 +294,20 @@ def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, t
 
 
 def spechub_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
-                        temperature=1.0, stream=None, out=None):
+                        temperature=1.0, stream=None, out=None, probabilities=True):
     """SpecHub verification of every node and the tree walk.  Returns the dict of output
-    tensors (see ``alloc_verify_outputs``); pass ``out`` to reuse buffers."""
+    tensors (see ``alloc_verify_outputs``); pass ``out`` to reuse buffers.  With
+    ``probabilities=False`` the library is given no beta / rate buffers (their tensors are left
+    untouched) and skips work that only they need."""
     return _verify("spechub", target_logits, draft_logits, draft_tokens, uniforms, tree, temperature,
-                   stream, out)
+                   stream, out, probabilities)
 
 
 def rrs_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
-                    without_replacement: bool, temperature=1.0, stream=None, out=None):
+                    without_replacement: bool, temperature=1.0, stream=None, out=None, probabilities=True):
     """RRS / RRSw verification of every node and the tree walk."""
     return _verify("rrsw" if without_replacement else "rrs", target_logits, draft_logits, draft_tokens,
-                   uniforms, tree, temperature, stream, out)
+                   uniforms, tree, temperature, stream, out, probabilities)
 
 
 def workspace_bytes(logits, tree: Tree, temperature=1.0) -> int:

@@ -620,6 +620,20 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             const float c = degenerate ? 0.f : 1.f / Q.sx;
             const float qa = invZq, rest = Q.sx * invZq;
             const int hubvec = hubtok >> 3, hubel = hubtok & 7;
+            const float px = prob_p(x), qx = prob_q(x);
+            if (!a.beta && !a.rate) {
+                // No probability is asked for: the first test needs scalars only, and if it accepts
+                // the transport sums decide nothing.
+                const bool acc1 = pair_xa ? accept_test(r1, px, qx, o.beta[0], true, o.status)
+                                          : accept_test(r1, fmaxf(__fsub_rn(px, qx), 0.f), c * qx, o.beta[0], true, o.status);
+                if (acc1) {
+                    o.accept_idx = pair_xa ? 0 : 1;
+                    o.token = x;
+                    if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
+                    break;
+                }
+                o.status = 0;  // the full path below sets the flags again
+            }
             // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
             float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
 #pragma unroll 2
@@ -651,7 +665,6 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             o.rate[1] = (degenerate ? 0.f : fmaxf(qa - S2, 0.f)) + fminf(hub_left, S1);
             o.rate[2] = R;
             if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
-            const float px = prob_p(x), qx = prob_q(x);
             bool acc1, acc2;
             if (pair_xa) {
                 acc1 = accept_test(r1, px, qx, o.beta[0], true, o.status);
@@ -694,6 +707,15 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
         } else {
             if (x1 < 0 || x1 >= a.vocab || x2 < 0 || x2 >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
+            if (!a.beta && !a.rate) {
+                // no probability asked for: an accepted first draft needs no sum at all
+                if (accept_test(r1, prob_p(x1), prob_q(x1), o.beta[0], true, o.status)) {
+                    o.accept_idx = 0;
+                    o.token = x1;
+                    break;
+                }
+                o.status = 0;
+            }
             // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
             const int x1vec = x1 >> 3, x1el = x1 & 7;
             float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;

@@ -293,6 +293,21 @@ __global__ void __launch_bounds__(512) verify_rows_kernel(RowArgs a) {
         const bool degenerate = !(Q.sx > 0.f);           // 1 - q(a) = 0
         const float c = degenerate ? 0.f : 1.f / Q.sx;     // q(a) / (1 - q(a))
         const float qa = invZq, rest = Q.sx * invZq;
+        if (!a.beta && !a.rate) {
+            // No probability is asked for: the first test needs scalars only, and if it accepts the
+            // transport sums decide nothing.
+            const float px0 = prob_p(x), qx0 = prob_q(x);
+            const bool acc0 = pair_xa ? accept_test(r1, px0, qx0, o.beta[0], true, o.status)
+                                      : accept_test(r1, fmaxf(__fsub_rn(px0, qx0), 0.f), c * qx0, o.beta[0], true, o.status);
+            if (acc0) {
+                o.accept_idx = pair_xa ? 0 : 1;
+                o.token = x;
+                if (degenerate) o.status |= SPECHUB_ST_DEGENERATE_Q;
+                if (threadIdx.x == 0) write_node(a, r, o);
+                return;
+            }
+            o.status = 0;
+        }
         // pass B: transport sums over ids != a (Section 4, Appendix B.1)
         float acc[3] = {0.f, 0.f, 0.f};  // S1, S2, R
         const int hubvec = hubtok / VW, hublane = hubtok % VW;
@@ -367,6 +382,16 @@ __global__ void __launch_bounds__(512) verify_rows_kernel(RowArgs a) {
             o.status = SPECHUB_ST_TOKEN_RANGE;
             if (threadIdx.x == 0) write_node(a, r, o);
             return;
+        }
+        if (!a.beta && !a.rate) {
+            // no probability asked for: an accepted first draft needs no sum at all
+            if (accept_test(r1, prob_p(x1), prob_q(x1), o.beta[0], true, o.status)) {
+                o.accept_idx = 0;
+                o.token = x1;
+                if (threadIdx.x == 0) write_node(a, r, o);
+                return;
+            }
+            o.status = 0;
         }
         // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
         float acc[2] = {0.f, 0.f};

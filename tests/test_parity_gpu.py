@@ -134,6 +134,30 @@ def test_lean_shapes(sh, V, split):
         sh.set_row_split(0)
 
 
+@pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (12344, "bf16"), (40000, "bf16")])
+def test_decisions_without_probabilities(sh, V, dtype):
+    """With no beta / rate buffers the library may stop after the first test; decisions, tokens,
+    hub and the walk must be the same as with them (bit for bit: same kernels, same arithmetic)."""
+    rng = np.random.default_rng(V + 17)
+    B, N = 6, 7
+    lp, lq = random_logits(rng, B, N, V, dtype, sigma=0.7)
+    un = random_uniforms(rng, B, N)
+    tp, tq, und = workloads.to_device(lp, dtype), workloads.to_device(lq, dtype), torch.from_numpy(un).cuda()
+    for paper in (False, True):
+        tree = sh.Tree.heap(N, leaves_sample=paper)
+        for m in METHODS:
+            d = gpu_draft(sh, m, tq, und, tree, 1.0)
+            full = parity.to_numpy(gpu_verify(sh, m, tp, tq, d["tokens"], und, tree, 1.0))
+            if m == "spechub":
+                lite = sh.spechub_verify_tree(tp, tq, d["tokens"], und, tree, 1.0, probabilities=False)
+            else:
+                lite = sh.rrs_verify_tree(tp, tq, d["tokens"], und, tree, m == "rrsw", 1.0, probabilities=False)
+            lite = parity.to_numpy(lite)
+            for k in ("accept_idx", "token", "hub", "n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+                np.testing.assert_array_equal(full[k], lite[k], err_msg="%s %s" % (m, k))
+            assert (full["accept_idx"] >= 0).any() and (full["accept_idx"] < 0).any()
+
+
 def test_peaked_rows_keep_precision(sh):
     """q close to one-hot: 1 - q(a) must come from a direct sum, not from 1 - q(a)."""
     rng = np.random.default_rng(5)
