@@ -284,6 +284,19 @@ def main():
     call_ms = {k: float(np.mean([a.elapsed_time(b) for a, b in v])) for k, v in ev_pairs.items()}
     verify_ms = call_ms["spechub_verify_tree"]
 
+    # ---- extra: SpecHub verification when the caller asks for decisions and tokens only ----
+    d0 = sh.spechub_draft_sample(tq, un, tree, cfg.temperature)
+    for _ in range(2):
+        sh.spechub_verify_tree(tp, tq, d0["tokens"], un, tree, cfg.temperature, out=outs["spechub"], probabilities=False)
+    barrier()
+    q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    q0.record(stream)
+    for _ in range(args.steps):
+        sh.spechub_verify_tree(tp, tq, d0["tokens"], un, tree, cfg.temperature, out=outs["spechub"], probabilities=False)
+    q1.record(stream)
+    barrier()
+    lite_ms = q0.elapsed_time(q1) / args.steps
+
     # ---- end to end: host buffers in, host results out, through the public API ----
     esz = 2 if cfg.dtype == "bf16" else 4
     h_tp = torch.empty(tp.shape, dtype=tp.dtype, pin_memory=True); h_tp.copy_(tp)
@@ -359,6 +372,10 @@ def main():
                 "spechub_verify_nodes_per_s": B * N / (verify_ms * 1e-3),
                 "spechub_verify_vocab_elements_per_s": B * N * V / (verify_ms * 1e-3),
                 "step_vocab_elements_per_s": nodes_per_step * V * args.steps / (ms * 1e-3),
+                "spechub_verify_without_probability_outputs": {
+                    "ms_per_launch": lite_ms, "nodes_per_s": B * N / (lite_ms * 1e-3),
+                    "note": "beta / rate not requested: rows whose first test accepts skip pass B; "
+                            "not part of `value`"},
             },
         }
         sfp = line["special_function_pipe"]
