@@ -33,10 +33,18 @@ METRIC = "tree-nodes verified/sec"
 UNIT = "nodes/s"
 METHODS = ("spechub", "rrs", "rrsw")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
-# profiles/, scaled from the captured batch to the workload's batch (traffic grows with the row
-# count).  Keyed by (API call, workload); absent = not captured for the current kernels.
-TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per (sequence, node) row, from the ncu capture
+# summarised in profiles/lean_kernels_c4_batch32.md (992 rows); a launch's traffic is this times its
+# row count (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not
+# captured for the current kernels.
+TRAFFIC_PER_ROW = {
+    ("spechub_draft_sample", "c4"): 272404880.0 / 992,
+    ("spechub_verify_tree", "c4"): 928103088.0 / 992,
+    ("rrs_draft_sample[rrs]", "c4"): 278853040.0 / 992,
+    ("rrs_verify_tree[rrs]", "c4"): 1316618304.0 / 992,
+    ("rrs_draft_sample[rrsw]", "c4"): 280562928.0 / 992,
+    ("rrs_verify_tree[rrsw]", "c4"): 1300669984.0 / 992,
+}
 
 
 def parse():
@@ -348,7 +356,9 @@ def main():
             ach = nbytes / (t_ms * 1e-3) / 1e9
             roof[name] = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
                           "frac": ach / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0,
-                          "traffic": TRAFFIC.get((name, cfg.name)), "alg_bytes_per_launch": nbytes,
+                          "traffic": (TRAFFIC_PER_ROW[(name, args.workload)] * B * N
+                                      if (name, args.workload) in TRAFFIC_PER_ROW and args.layout == "dense" else None),
+                          "alg_bytes_per_launch": nbytes,
                           "ms_per_launch": t_ms, "share_of_step": t_ms / total_call_ms}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
