@@ -22,6 +22,11 @@ from .oracle import (  # noqa: F401
     hub,
     inv_cdf,
     rrs_draft,
+    rrs_k_draft,
+    rrs_k_draft_batch,
+    rrs_k_residual,
+    rrs_k_verify,
+    rrs_k_verify_batch,
     rrs_residual,
     rrs_verify,
     softmax,
@@ -30,4 +35,5 @@ from .oracle import (  # noqa: F401
     spechub_verify,
     verify_batch,
     walk,
+    walk_k,
 )

@@ -102,6 +102,23 @@ def _load():
         lib.orc_walk.restype = None
         lib.orc_walk.argtypes = [_ip, _ip, ctypes.c_int, ctypes.c_int, _ip, _bp, ctypes.c_int,
                                  _ip, _ip, _ip, _ip]
+        lib.orc_rrs_k_draft.restype = ctypes.c_uint
+        lib.orc_rrs_k_draft.argtypes = [_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int, _dp, _ip, _dp]
+        lib.orc_rrs_k_verify.restype = None
+        lib.orc_rrs_k_verify.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_int, _ip, _dp, ctypes.c_double,
+                                         ctypes.c_int, _ip, _ip, _dp, _dp, _dp, _dp, _up]
+        lib.orc_rrs_k_residual.restype = None
+        lib.orc_rrs_k_residual.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_int, _ip, ctypes.c_int, _dp]
+        lib.orc_rrs_k_draft_batch.restype = None
+        lib.orc_rrs_k_draft_batch.argtypes = [ctypes.c_int, ctypes.c_int, _fp, _fp, ctypes.c_int, ctypes.c_int,
+                                              ctypes.c_int, _fp, _ip, _dp, _up]
+        lib.orc_rrs_k_verify_batch.restype = None
+        lib.orc_rrs_k_verify_batch.argtypes = [ctypes.c_int, ctypes.c_int, _fp, _fp, _fp, ctypes.c_int,
+                                               ctypes.c_int, ctypes.c_int, _bp, _ip, _fp, _ip, _ip, _dp, _dp,
+                                               _dp, _dp, _up]
+        lib.orc_walk_k.restype = None
+        lib.orc_walk_k.argtypes = [ctypes.c_int, _ip, _ip, ctypes.c_int, ctypes.c_int, _ip, _bp, ctypes.c_int,
+                                   _ip, _ip, _ip, _ip]
         lib.orc_node_size.restype = ctypes.c_size_t
         assert lib.orc_node_size() == NODE_DTYPE.itemsize, (lib.orc_node_size(), NODE_DTYPE.itemsize)
         _lib = lib
@@ -290,4 +307,88 @@ def walk(accept_idx, token, levels, child=None, node_kind=None):
     _load().orc_walk(_ptr(ai, _ip), _ptr(tk, _ip), B, N, _ptr(ch, _ip) if ch is not None else None,
                      _ptr(nk, _bp) if nk is not None else None, int(levels), _ptr(na, _ip),
                      _ptr(ne, _ip), _ptr(pn, _ip), _ptr(pt, _ip))
+    return dict(n_accepted=na, n_emitted=ne, path_nodes=pn, path_tokens=pt)
+
+
+# ---- Algorithm 1 for general k ------------------------------------------------------------------
+
+def rrs_k_draft(q, k, without_replacement, u):
+    """k drafts from q (independent, or without replacement).  Returns (tokens[k], margin[k], status)."""
+    q = _f64(q)
+    u = _f64(u)
+    tk = np.empty(k, np.int32)
+    mg = np.empty(k, np.float64)
+    st = _load().orc_rrs_k_draft(_ptr(q, _dp), q.shape[0], int(k), int(bool(without_replacement)),
+                                 _ptr(u, _dp), _ptr(tk, _ip), _ptr(mg, _dp))
+    return tk, mg, int(st)
+
+
+def rrs_k_verify(p, q, tokens, r, u_res, without_replacement):
+    """Algorithm 1 on one node with k = len(tokens) drafts.  Returns a dict."""
+    p, q, r = _f64(p), _f64(q), _f64(r)
+    tk = _i32(tokens)
+    k = tk.shape[0]
+    ai, tok, st = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_uint32()
+    beta, rate = np.empty(k), np.empty(k + 1)
+    margin, cond = np.empty(k + 1), np.empty(k)
+    _load().orc_rrs_k_verify(_ptr(p, _dp), _ptr(q, _dp), p.shape[0], k, _ptr(tk, _ip), _ptr(r, _dp),
+                             float(u_res), int(bool(without_replacement)), ctypes.byref(ai),
+                             ctypes.byref(tok), _ptr(beta, _dp), _ptr(rate, _dp), _ptr(margin, _dp),
+                             _ptr(cond, _dp), ctypes.byref(st))
+    return dict(accept_idx=ai.value, token=tok.value, beta=beta, rate=rate, margin=margin, cond=cond,
+                status=st.value)
+
+
+def rrs_k_residual(p, q, tokens, without_replacement):
+    p, q = _f64(p), _f64(q)
+    tk = _i32(tokens)
+    w = np.empty_like(p)
+    _load().orc_rrs_k_residual(_ptr(p, _dp), _ptr(q, _dp), p.shape[0], tk.shape[0], _ptr(tk, _ip),
+                               int(bool(without_replacement)), _ptr(w, _dp))
+    return w
+
+
+def rrs_k_draft_batch(k, without_replacement, draft_logits, temperature, uniforms):
+    lq = _f32(draft_logits)
+    B, N, V = lq.shape
+    un = _f32(uniforms)
+    assert un.shape == (B, N, 2 * k + 1)
+    t = _temps(temperature, B)
+    tokens = np.empty((B, N, k), np.int32)
+    margin = np.empty((B, N, k), np.float64)
+    status = np.zeros((B, N), np.uint32)
+    _load().orc_rrs_k_draft_batch(int(k), int(bool(without_replacement)), _ptr(lq, _fp), _ptr(t, _fp), B, N, V,
+                                  _ptr(un, _fp), _ptr(tokens, _ip), _ptr(margin, _dp), _ptr(status, _up))
+    return dict(tokens=tokens, margin=margin, status=status)
+
+
+def rrs_k_verify_batch(k, without_replacement, target_logits, draft_logits, temperature, draft_tokens,
+                       uniforms, node_kind=None):
+    lp, lq = _f32(target_logits), _f32(draft_logits)
+    B, N, V = lp.shape
+    un, tk = _f32(uniforms), _i32(draft_tokens)
+    assert un.shape == (B, N, 2 * k + 1) and tk.shape == (B, N, k)
+    t = _temps(temperature, B)
+    nk = None if node_kind is None else np.ascontiguousarray(node_kind, dtype=np.uint8)
+    out = dict(accept_idx=np.empty((B, N), np.int32), token=np.empty((B, N), np.int32),
+               beta=np.empty((B, N, k)), rate=np.empty((B, N, k + 1)), margin=np.empty((B, N, k + 1)),
+               cond=np.empty((B, N, k)), status=np.zeros((B, N), np.uint32))
+    _load().orc_rrs_k_verify_batch(int(k), int(bool(without_replacement)), _ptr(lp, _fp), _ptr(lq, _fp),
+                                   _ptr(t, _fp), B, N, V, _ptr(nk, _bp) if nk is not None else None,
+                                   _ptr(tk, _ip), _ptr(un, _fp), _ptr(out["accept_idx"], _ip),
+                                   _ptr(out["token"], _ip), _ptr(out["beta"], _dp), _ptr(out["rate"], _dp),
+                                   _ptr(out["margin"], _dp), _ptr(out["cond"], _dp), _ptr(out["status"], _up))
+    return out
+
+
+def walk_k(k, accept_idx, token, levels, child=None, node_kind=None):
+    ai, tk = _i32(accept_idx), _i32(token)
+    B, N = ai.shape
+    ch = None if child is None else _i32(child)
+    nk = None if node_kind is None else np.ascontiguousarray(node_kind, dtype=np.uint8)
+    na, ne = np.empty(B, np.int32), np.empty(B, np.int32)
+    pn, pt = np.empty((B, levels), np.int32), np.empty((B, levels), np.int32)
+    _load().orc_walk_k(int(k), _ptr(ai, _ip), _ptr(tk, _ip), B, N, _ptr(ch, _ip) if ch is not None else None,
+                       _ptr(nk, _bp) if nk is not None else None, int(levels), _ptr(na, _ip), _ptr(ne, _ip),
+                       _ptr(pn, _ip), _ptr(pt, _ip))
     return dict(n_accepted=na, n_emitted=ne, path_nodes=pn, path_tokens=pt)

@@ -522,4 +522,213 @@ void orc_walk(const int32_t *accept_idx, const int32_t *token, int B, int N, con
     }
 }
 
+
+/* ======================= Algorithm 1 for general k ============================
+ * The paper states Algorithm 1 for k candidates (its ternary trees and the
+ * 10-draft acceptance decay of Appendix C use k > 2).  Layout of the uniforms
+ * of a node: (u_d1..u_dk, r_1..r_k, u_res), 2k+1 values.
+ *
+ * Draft step: k samples from q independently (RRS) or without replacement
+ * (RRSw: after each draw q(x_i) <- 0 and q is renormalised). */
+unsigned orc_rrs_k_draft(const double *q, int V, int k, int without_replacement, const double *u,
+                         int32_t *tokens, double *margin) {
+    unsigned st = 0u;
+    double *w = (double *)malloc(sizeof(double) * (size_t)V);
+    memcpy(w, q, sizeof(double) * (size_t)V);
+    for (int i = 0; i < k; ++i) {
+        margin[i] = INFINITY;
+        int x = orc_inv_cdf(w, V, u[i], NULL, &margin[i]);
+        if (x < 0) {              /* nothing left to draw from: lowest id not drawn yet */
+            st |= ORC_DEGENERATE_Q;
+            margin[i] = INFINITY;
+            for (x = 0; x < V; ++x) {
+                int used = 0;
+                for (int j = 0; j < i; ++j) used |= (tokens[j] == x);
+                if (!used) break;
+            }
+            if (x >= V) x = 0;
+        }
+        tokens[i] = x;
+        if (without_replacement) w[x] = 0.0;   /* the draw normalises by the remaining mass */
+    }
+    free(w);
+    return st;
+}
+
+/* Verification of k drafts, Algorithm 1 step by step:
+ *   for i = 1..k: accept x_i iff r_i < p(x_i)/q(x_i) (strict, multiplicative; q(x_i) = 0 rejects);
+ *                 else p <- norm(max(p - q, 0)); [RRSw: q(x_i) <- 0, q <- norm(q)]
+ *   return x ~ p.
+ * Outputs: accept_idx in {-1, 0..k-1}; token; beta[k] (acceptance probability of test i, given
+ * that it is reached); rate[k+1] (mass of accepting at stage i for these drafts -- unconditional
+ * for RRS stage 1 only -- and of rejecting all); margin[k+1]; cond[k]; status.
+ * If a residual has no mass (p = q so far) the draw falls back to the original p with
+ * ORC_ZERO_RESIDUAL, and later tests have beta = 0. */
+void orc_rrs_k_verify(const double *p0, const double *q0, int V, int k, const int32_t *x,
+                      const double *r, double u_res, int without_replacement, int32_t *accept_idx,
+                      int32_t *token, double *beta, double *rate, double *margin, double *cond,
+                      uint32_t *status) {
+    *accept_idx = -1; *token = -1; *status = 0u;
+    for (int i = 0; i < k; ++i) { beta[i] = 0.0; cond[i] = 0.0; margin[i] = INFINITY; rate[i] = 0.0; }
+    margin[k] = INFINITY; rate[k] = 0.0;
+    for (int i = 0; i < k; ++i)
+        if (x[i] < 0 || x[i] >= V) { *status |= ORC_TOKEN_RANGE; return; }
+    double *p = (double *)malloc(sizeof(double) * (size_t)V * 3), *q = p + V, *mag = q + V;
+    memcpy(p, p0, sizeof(double) * (size_t)V);
+    memcpy(q, q0, sizeof(double) * (size_t)V);
+    for (int y = 0; y < V; ++y) mag[y] = p0[y];     /* |terms| of p(y), for cond[] only */
+    double mass = 1.0;       /* probability of reaching the current stage with these drafts' stages */
+    double amp = 1.0;        /* growth of the relative error through the normalisations          */
+    int accepted = 0, alive = 1;
+    for (int i = 0; i < k; ++i) {
+        int performed = alive && !accepted;
+        int xi = x[i];
+        double N = p[xi], D = q[xi];
+        beta[i] = (alive && D > 0.0) ? dmin(N / D, 1.0) : 0.0;
+        cond[i] = (alive && D > 0.0) ? (mag[xi] * amp + beta[i] * D) / D : 0.0;
+        /* mass accepted at this stage: sum_y min(p, q) of the current pair, times the mass so far */
+        nsum acc; ns_init(&acc);
+        if (alive) for (int y = 0; y < V; ++y) ns_add(&acc, dmin(p[y], q[y]));
+        rate[i] = alive ? mass * ns_val(&acc) : 0.0;
+        if (performed) {
+            if (!(D > 0.0)) { *status |= ORC_ZERO_MASS_DRAFT; }
+            else {
+                margin[i] = fabs(r[i] - N / D);
+                if (r[i] * D < N) { accepted = 1; *accept_idx = i; *token = xi; }
+            }
+        }
+        if (!alive) continue;
+        /* p <- norm(max(p - q, 0)) */
+        nsum a; ns_init(&a);
+        double nA = 0.0;
+        for (int y = 0; y < V; ++y) {
+            double d = p[y] - q[y];
+            if (d > 0.0) { mag[y] = mag[y] + q[y]; nA += mag[y]; p[y] = d; } else { p[y] = 0.0; mag[y] = 0.0; }
+            ns_add(&a, p[y]);
+        }
+        double A = ns_val(&a);
+        mass *= A;
+        if (A > 0.0) {
+            for (int y = 0; y < V; ++y) { p[y] /= A; mag[y] /= A; }
+            amp += nA / A;
+        } else {
+            alive = 0;
+        }
+        if (without_replacement && alive) {
+            q[xi] = 0.0;
+            nsum d; ns_init(&d);
+            for (int y = 0; y < V; ++y) ns_add(&d, q[y]);
+            double den = ns_val(&d);
+            if (den > 0.0) { for (int y = 0; y < V; ++y) q[y] /= den; }
+            else { if (!accepted) *status |= ORC_DEGENERATE_Q; }
+        }
+    }
+    rate[k] = mass;
+    if (!accepted) {
+        int tok = alive ? orc_inv_cdf(p, V, u_res, NULL, &margin[k]) : -1;
+        if (tok < 0) {
+            *status |= ORC_ZERO_RESIDUAL;
+            tok = orc_inv_cdf(p0, V, u_res, NULL, &margin[k]);
+        }
+        *token = tok;
+    }
+    free(p);
+}
+
+/* Residual weights after all k drafts were rejected (unnormalised); 0 mass if none. */
+void orc_rrs_k_residual(const double *p0, const double *q0, int V, int k, const int32_t *x,
+                        int without_replacement, double *w) {
+    double *q = (double *)malloc(sizeof(double) * (size_t)V);
+    memcpy(w, p0, sizeof(double) * (size_t)V);
+    memcpy(q, q0, sizeof(double) * (size_t)V);
+    for (int i = 0; i < k; ++i) {
+        nsum a; ns_init(&a);
+        for (int y = 0; y < V; ++y) { w[y] = dmax(w[y] - q[y], 0.0); ns_add(&a, w[y]); }
+        double A = ns_val(&a);
+        if (!(A > 0.0)) break;
+        for (int y = 0; y < V; ++y) w[y] /= A;
+        if (without_replacement) {
+            q[x[i]] = 0.0;
+            nsum d; ns_init(&d);
+            for (int y = 0; y < V; ++y) ns_add(&d, q[y]);
+            double den = ns_val(&d);
+            if (den > 0.0) for (int y = 0; y < V; ++y) q[y] /= den;
+        }
+    }
+    free(q);
+}
+
+void orc_rrs_k_draft_batch(int k, int without_replacement, const float *draft_logits,
+                           const float *temperature, int B, int N, int V, const float *uniforms,
+                           int32_t *tokens, double *margin, uint32_t *status) {
+    double *q = (double *)malloc(sizeof(double) * (size_t)V);
+    double u[64];
+    const int nu = 2 * k + 1;
+    for (long r = 0; r < (long)B * N; ++r) {
+        for (int i = 0; i < k; ++i) { tokens[r * k + i] = -1; margin[r * k + i] = INFINITY; }
+        unsigned st = orc_softmax(draft_logits + (size_t)r * V, V, (double)temperature[r / N], q);
+        if (st) { status[r] = st; continue; }
+        for (int i = 0; i < k; ++i) u[i] = (double)uniforms[(size_t)r * nu + i];
+        status[r] = orc_rrs_k_draft(q, V, k, without_replacement, u, tokens + r * k, margin + r * k);
+    }
+    free(q);
+}
+
+void orc_rrs_k_verify_batch(int k, int without_replacement, const float *target_logits,
+                            const float *draft_logits, const float *temperature, int B, int N, int V,
+                            const uint8_t *node_kind, const int32_t *draft_tokens,
+                            const float *uniforms, int32_t *accept_idx, int32_t *token, double *beta,
+                            double *rate, double *margin, double *cond, uint32_t *status) {
+    double *p = (double *)malloc(sizeof(double) * (size_t)V * 2), *q = p + V;
+    double rr[64];
+    const int nu = 2 * k + 1;
+    for (long r = 0; r < (long)B * N; ++r) {
+        int n = (int)(r % N);
+        const float *u = uniforms + (size_t)r * nu;
+        accept_idx[r] = -1; token[r] = -1; status[r] = 0u;
+        for (int i = 0; i < k; ++i) { beta[r * k + i] = 0.0; cond[r * k + i] = 0.0; }
+        for (int i = 0; i <= k; ++i) { rate[r * (k + 1) + i] = 0.0; margin[r * (k + 1) + i] = INFINITY; }
+        double T = (double)temperature[r / N];
+        unsigned st = orc_softmax(target_logits + (size_t)r * V, V, T, p);
+        if (st) { status[r] = st; continue; }
+        if (node_kind && node_kind[n] == 1) {
+            token[r] = orc_inv_cdf(p, V, u[2 * k], NULL, &margin[r * (k + 1) + k]);
+            rate[r * (k + 1) + k] = 1.0;
+            continue;
+        }
+        st = orc_softmax(draft_logits + (size_t)r * V, V, T, q);
+        if (st) { status[r] = st; continue; }
+        for (int i = 0; i < k; ++i) rr[i] = (double)u[k + i];
+        orc_rrs_k_verify(p, q, V, k, draft_tokens + r * k, rr, (double)u[2 * k], without_replacement,
+                         accept_idx + r, token + r, beta + r * k, rate + r * (k + 1),
+                         margin + r * (k + 1), cond + r * k, status + r);
+    }
+    free(p);
+}
+
+/* Tree walk with k children per node: child[n][i] (NULL = complete k-ary tree in level order,
+ * child i of n is k*n + 1 + i). */
+void orc_walk_k(int k, const int32_t *accept_idx, const int32_t *token, int B, int N,
+                const int32_t *child, const uint8_t *node_kind, int levels, int32_t *n_accepted,
+                int32_t *n_emitted, int32_t *path_nodes, int32_t *path_tokens) {
+    for (int b = 0; b < B; ++b) {
+        int32_t *pn = path_nodes + (size_t)b * levels, *pt = path_tokens + (size_t)b * levels;
+        for (int i = 0; i < levels; ++i) { pn[i] = -1; pt[i] = -1; }
+        int n = 0, acc = 0, emitted = 0;
+        for (int step = 0; step < levels && n >= 0 && n < N; ++step) {
+            long r = (long)b * N + n;
+            pn[step] = n;
+            if (token[r] < 0) break;
+            pt[step] = token[r];
+            ++emitted;
+            if (node_kind && node_kind[n] == 1) break;
+            int idx = accept_idx[r];
+            if (idx < 0) break;
+            ++acc;
+            n = child ? child[k * n + idx] : k * n + 1 + idx;
+        }
+        n_accepted[b] = acc; n_emitted[b] = emitted;
+    }
+}
+
 size_t orc_node_size(void) { return sizeof(orc_node); }
