@@ -34,7 +34,11 @@
  *     second acceptance test performed at the node; u_res the residual (or
  *     leaf) draw.  draft_tokens are int32 [batch][nodes][2]; per-node outputs
  *     are [batch][nodes] (row-major), with 2 or 3 trailing entries where
- *     stated.
+ *     stated.  With k drafts per node (RRS / RRSw only) the same layouts
+ *     hold with k in place of 2: uniforms [..][2k+1] = (u_d1..u_dk, r_1..r_k,
+ *     u_res), draft_tokens [..][k], beta [..][k], rate [..][k+1], child
+ *     [nodes][k] (NULL = complete k-ary tree, child i of n is k*n + 1 + i),
+ *     accept_idx in {-1, 0..k-1}.
  *   - Sampling from a non-negative weight vector w with a uniform u always
  *     means: the lowest token id j whose inclusive prefix sum over ascending
  *     ids exceeds u * sum(w); zero-weight ids are never returned.
@@ -52,6 +56,7 @@ extern "C" {
 #endif
 
 #define SPECHUB_ABI_VERSION 1
+#define SPECHUB_MAX_K 8 /* most drafts per node the RRS / RRSw entry points take */
 
 /* return codes */
 #define SPECHUB_OK 0
@@ -94,7 +99,8 @@ typedef struct spechub_desc {
     int32_t batch;        /* sequences B                                                     */
     int32_t nodes;        /* tree nodes per sequence N, level order, node 0 = root           */
     int32_t vocab;        /* V >= 2                                                          */
-    int32_t k;            /* drafts per node; must be 2 (Section 4)                          */
+    int32_t k;            /* drafts per node: 2 for SpecHub (Section 4); 2..SPECHUB_MAX_K for
+                             RRS / RRSw (Algorithm 1 is stated for k candidates)             */
     int32_t dtype;        /* SPECHUB_F32 or SPECHUB_BF16 logits                              */
     int32_t levels;       /* longest root-to-leaf path in nodes; bounds the walk, row length
                              of the path outputs                                             */
@@ -155,7 +161,10 @@ int spechub_draft_sample(const spechub_desc *desc, const void *draft_logits, con
  * Draft step of RRS / RRSw (Algorithm 1, "Generate k samples ... independently
  * or without replacement from q").  x1 is drawn from q with u_d1; x2 from q
  * with u_d2 (without_replacement = 0) or from q with q(x1) set to 0
- * (without_replacement = 1).  Arguments as above.
+ * (without_replacement = 1).  Arguments as above.  For desc->k > 2 draw i uses
+ * u_di and, without replacement, q with q(x1..x_{i-1}) set to 0; if nothing is
+ * left to draw from, the lowest id not drawn yet is returned with
+ * SPECHUB_ST_DEGENERATE_Q.
  */
 int rrs_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
                      int without_replacement, int32_t *draft_tokens, uint32_t *status, void *stream);
@@ -197,6 +206,11 @@ int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
  *   max(max(p - q, 0) - A1 q1, 0).
  * rate = (sum min(p,q), A1 - W2, W2), W2 the mass of that last residual (for
  * RRSw the last two are for the given x1).  hub is written as -1.
+ * For desc->k > 2 the loop of Algorithm 1 runs over all k drafts: with P_0 = p,
+ * m_0 = 1, draft x_j is accepted iff r_j m_{j-1} q_j(x_j) < P_{j-1}(x_j), where
+ * q_j = q (RRS) or q with q(x_1..x_{j-1}) zeroed and renormalised (RRSw),
+ * P_j = max(P_{j-1} - m_{j-1} q_j, 0) and m_j = sum P_j; the residual token is
+ * drawn from P_k; rate[j] = m_j - m_{j+1} (j < k), rate[k] = m_k.
  */
 int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
                     const int32_t *draft_tokens, const float *uniforms, int without_replacement,

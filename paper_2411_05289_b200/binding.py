@@ -138,8 +138,9 @@ class Tree:
     (None = complete binary tree in heap order, every node verifies)."""
 
     levels: int
-    child: Optional[torch.Tensor] = None      # int32 [nodes][2]
+    child: Optional[torch.Tensor] = None      # int32 [nodes][k]
     node_kind: Optional[torch.Tensor] = None  # uint8 [nodes]
+    k: int = 2                                # drafts (children) per node; > 2 for RRS / RRSw only
 
     @staticmethod
     def heap(nodes: int, leaves_sample: bool = False, device="cuda") -> "Tree":
@@ -154,6 +155,20 @@ class Tree:
             kind[nodes // 2:] = 1
             kind = kind.to(device)
         return Tree(levels=d, child=None, node_kind=kind)
+
+    @staticmethod
+    def kary(k: int, levels: int, leaves_sample: bool = False, device="cuda") -> "Tree":
+        """Complete k-ary tree with `levels` levels in level order ((k^levels - 1)/(k - 1) nodes)."""
+        nodes = (k ** levels - 1) // (k - 1)
+        kind = None
+        if leaves_sample:
+            kind = torch.zeros(nodes, dtype=torch.uint8)
+            kind[(k ** (levels - 1) - 1) // (k - 1):] = 1
+            kind = kind.to(device)
+        return Tree(levels=levels, child=None, node_kind=kind, k=k)
+
+    def nodes_of_complete_tree(self) -> int:
+        return (self.k ** self.levels - 1) // (self.k - 1)
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -180,7 +195,7 @@ def _desc(logits: torch.Tensor, tree: Tree, temperature) -> tuple:
     d = _Desc()
     d.struct_size = ctypes.sizeof(_Desc)
     d.version = ABI_VERSION
-    d.batch, d.nodes, d.vocab, d.k = B, N, V, 2
+    d.batch, d.nodes, d.vocab, d.k = B, N, V, tree.k
     d.dtype = dt
     d.levels = tree.levels
     d.stride_seq = logits.stride(0) if B > 1 else max(logits.stride(0), (N - 1) * logits.stride(1) + V)
@@ -197,8 +212,8 @@ def _desc(logits: torch.Tensor, tree: Tree, temperature) -> tuple:
         d.temperature = float(temperature)
         d.temperature_per_seq = None
     if tree.child is not None:
-        if tree.child.dtype != torch.int32 or tuple(tree.child.shape) != (N, 2) or not tree.child.is_contiguous():
-            raise ValueError("child must be a contiguous int32 [nodes][2] tensor")
+        if tree.child.dtype != torch.int32 or tuple(tree.child.shape) != (N, tree.k) or not tree.child.is_contiguous():
+            raise ValueError("child must be a contiguous int32 [nodes][k] tensor")
         d.child = tree.child.data_ptr()
     if tree.node_kind is not None:
         if tree.node_kind.dtype != torch.uint8 or tuple(tree.node_kind.shape) != (N,):
@@ -213,14 +228,21 @@ def _same_layout(a: torch.Tensor, b: torch.Tensor):
         raise ValueError("target and draft logits must share shape, dtype, strides and device")
 
 
-def _check_uniforms(u, B, N, dev):
-    if u.dtype != torch.float32 or tuple(u.shape) != (B, N, 5) or not u.is_contiguous() or u.device != dev:
-        raise ValueError("uniforms must be a contiguous float32 [batch][nodes][5] tensor on the logits' device")
+def _check_uniforms(u, B, N, dev, k=2):
+    if (u.dtype != torch.float32 or tuple(u.shape) != (B, N, 2 * k + 1) or not u.is_contiguous()
+            or u.device != dev):
+        raise ValueError("uniforms must be a contiguous float32 [batch][nodes][2k+1] tensor on the logits' device")
+
+
+def _need_k2(tree):
+    if tree.k != 2:
+        raise ValueError("SpecHub takes exactly two drafts per node")
 
 
 def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
     """Draw the k = 2 SpecHub drafts of every node.  Returns dict(tokens, hub, prob, status)."""
     lib = load_library()
+    _need_k2(tree)
     d, keep = _desc(draft_logits, tree, temperature)
     B, N, _ = draft_logits.shape
     dev = draft_logits.device
@@ -236,13 +258,13 @@ def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, st
 
 def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bool, temperature=1.0,
                      stream=None):
-    """Draw the k = 2 RRS / RRSw drafts of every node.  Returns dict(tokens, status)."""
+    """Draw the k = tree.k RRS / RRSw drafts of every node.  Returns dict(tokens, status)."""
     lib = load_library()
     d, keep = _desc(draft_logits, tree, temperature)
     B, N, _ = draft_logits.shape
     dev = draft_logits.device
-    _check_uniforms(uniforms, B, N, dev)
-    tokens = torch.empty((B, N, 2), dtype=torch.int32, device=dev)
+    _check_uniforms(uniforms, B, N, dev, tree.k)
+    tokens = torch.empty((B, N, tree.k), dtype=torch.int32, device=dev)
     status = torch.empty((B, N), dtype=torch.int32, device=dev)
     _check(lib.rrs_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
                                 int(bool(without_replacement)), _ptr(tokens), _ptr(status),
@@ -250,14 +272,14 @@ def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bo
     return dict(tokens=tokens, status=status)
 
 
-def alloc_verify_outputs(B, N, levels, dev):
+def alloc_verify_outputs(B, N, levels, dev, k=2):
     """Device buffers for one verify call (reusable across calls of the same shape)."""
     return dict(
         accept_idx=torch.empty((B, N), dtype=torch.int32, device=dev),
         token=torch.empty((B, N), dtype=torch.int32, device=dev),
         hub=torch.empty((B, N), dtype=torch.int32, device=dev),
-        beta=torch.empty((B, N, 2), dtype=torch.float32, device=dev),
-        rate=torch.empty((B, N, 3), dtype=torch.float32, device=dev),
+        beta=torch.empty((B, N, k), dtype=torch.float32, device=dev),
+        rate=torch.empty((B, N, k + 1), dtype=torch.float32, device=dev),
         status=torch.empty((B, N), dtype=torch.int32, device=dev),
         n_accepted=torch.empty((B,), dtype=torch.int32, device=dev),
         n_emitted=torch.empty((B,), dtype=torch.int32, device=dev),
@@ -273,12 +295,14 @@ def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, t
     d, keep = _desc(target_logits, tree, temperature)
     B, N, _ = target_logits.shape
     dev = target_logits.device
-    _check_uniforms(uniforms, B, N, dev)
-    if (draft_tokens.dtype != torch.int32 or tuple(draft_tokens.shape) != (B, N, 2)
+    if method == "spechub":
+        _need_k2(tree)
+    _check_uniforms(uniforms, B, N, dev, tree.k)
+    if (draft_tokens.dtype != torch.int32 or tuple(draft_tokens.shape) != (B, N, tree.k)
             or not draft_tokens.is_contiguous() or draft_tokens.device != dev):
-        raise ValueError("draft_tokens must be a contiguous int32 [batch][nodes][2] tensor")
+        raise ValueError("draft_tokens must be a contiguous int32 [batch][nodes][k] tensor")
     if out is None:
-        out = alloc_verify_outputs(B, N, tree.levels, dev)
+        out = alloc_verify_outputs(B, N, tree.levels, dev, tree.k)
     no = _NodeOut(*[out[k].data_ptr() if (probabilities or k not in ("beta", "rate")) else None
                     for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
     so = _SeqOut(*[out[k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])

@@ -8,6 +8,7 @@
 #include "spechub_common.cuh"
 #include "spechub_stream.cuh"
 #include "spechub_lean.cuh"
+#include "spechub_kary.cuh"
 
 namespace {
 
@@ -17,7 +18,7 @@ int check_desc(const spechub_desc *d) {
     if (!d) return SPECHUB_ERR_NULL;
     if (d->struct_size != sizeof(spechub_desc) || d->version != SPECHUB_ABI_VERSION)
         return SPECHUB_ERR_VERSION;
-    if (d->batch < 0 || d->nodes < 1 || d->vocab < 2 || d->k != 2 || d->levels < 1)
+    if (d->batch < 0 || d->nodes < 1 || d->vocab < 2 || d->k < 2 || d->k > SPECHUB_MAX_K || d->levels < 1)
         return SPECHUB_ERR_SHAPE;
     if (d->dtype != SPECHUB_F32 && d->dtype != SPECHUB_BF16) return SPECHUB_ERR_DTYPE;
     if (d->stride_node < d->vocab) return SPECHUB_ERR_STRIDE;
@@ -131,7 +132,18 @@ int draft_common(const spechub_desc *d, const void *draft_logits, const float *u
     const int th = threads_for(d);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, draft_logits);
-    if (lean_ok(d, al)) {
+    if (d->k > 2) {
+        if (method == kSpecHub) return SPECHUB_ERR_SHAPE;
+        KaryArgs ka;
+        ka.r = a; ka.k = d->k; ka.without_replacement = (method == kRRSw);
+        if (d->dtype == SPECHUB_BF16) {
+            if (al) kary_draft_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(ka);
+            else kary_draft_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(ka);
+        } else {
+            if (al) kary_draft_kernel<float, true><<<rows, th, 0, s>>>(ka);
+            else kary_draft_kernel<float, false><<<rows, th, 0, s>>>(ka);
+        }
+    } else if (lean_ok(d, al)) {
         const int lrc = launch_lean_draft(method, lean_split(d), a, rows, s);
         if (lrc != SPECHUB_OK) return lrc;
     } else if (d->dtype == SPECHUB_BF16) {
@@ -183,7 +195,18 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
     const int th = threads_for(d);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool al = rows_aligned(d, target_logits) && rows_aligned(d, draft_logits);
-    if (lean_ok(d, al)) {
+    if (d->k > 2) {
+        if (method == kSpecHub) return SPECHUB_ERR_SHAPE;
+        KaryArgs ka;
+        ka.r = a; ka.k = d->k; ka.without_replacement = (method == kRRSw);
+        if (d->dtype == SPECHUB_BF16) {
+            if (al) kary_verify_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(ka);
+            else kary_verify_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(ka);
+        } else {
+            if (al) kary_verify_kernel<float, true><<<rows, th, 0, s>>>(ka);
+            else kary_verify_kernel<float, false><<<rows, th, 0, s>>>(ka);
+        }
+    } else if (lean_ok(d, al)) {
         const int lrc = launch_lean_verify(method, lean_split(d), a, rows, s);
         if (lrc != SPECHUB_OK) return lrc;
     } else if (method == kSpecHub) launch_verify<kSpecHub>(d, a, al, rows, th, s);
@@ -204,7 +227,13 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
         w.batch = d->batch;
         w.nodes = d->nodes;
         w.levels = d->levels;
-        walk_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(w);
+        if (d->k > 2) {
+            WalkKArgs wk;
+            wk.w = w; wk.k = d->k;
+            walk_k_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(wk);
+        } else {
+            walk_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(w);
+        }
         lrc = launch_status();
     }
     return lrc;
@@ -257,7 +286,7 @@ const char *spechub_status_string(int code) {
         case SPECHUB_OK: return "ok";
         case SPECHUB_ERR_NULL: return "a required pointer is NULL";
         case SPECHUB_ERR_VERSION: return "descriptor struct_size/version mismatch";
-        case SPECHUB_ERR_SHAPE: return "bad shape: need batch >= 0, nodes >= 1, vocab >= 2, k == 2, levels >= 1, valid flags";
+        case SPECHUB_ERR_SHAPE: return "bad shape: need batch >= 0, nodes >= 1, vocab >= 2, 2 <= k <= 8 (k == 2 for SpecHub), levels >= 1, valid flags";
         case SPECHUB_ERR_DTYPE: return "dtype must be SPECHUB_F32 or SPECHUB_BF16";
         case SPECHUB_ERR_STRIDE: return "strides too small for the given shape";
         case SPECHUB_ERR_TEMPERATURE: return "temperature must be finite and > 0";

@@ -57,7 +57,8 @@ def test_host_side_argument_checks_need_no_gpu():
 
     fake = ctypes.c_void_p(16)  # never dereferenced: every call below is rejected on the host
     call = lambda d: lib.spechub_draft_sample(ctypes.byref(d), fake, fake, fake, None, None, None, None)
-    assert call(desc(k=3)) == -3
+    assert call(desc(k=3)) == -3   # SpecHub takes exactly two drafts
+    assert call(desc(k=9)) == -3
     assert call(desc(vocab=1)) == -3
     assert call(desc(nodes=0)) == -3
     assert call(desc(batch=-1)) == -3

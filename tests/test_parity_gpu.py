@@ -232,7 +232,7 @@ def test_argument_errors(sh):
     call = lambda dd: lib.spechub_draft_sample(ctypes.byref(dd), vp(x.data_ptr()), vp(un.data_ptr()),
                                                vp(tok.data_ptr()), None, None, None, None)
     assert call(d) == 0
-    for field, val, code in [("k", 3, -3), ("vocab", 1, -3), ("dtype", 7, -4), ("version", 9, -2),
+    for field, val, code in [("k", 3, -3), ("k", 1, -3), ("vocab", 1, -3), ("dtype", 7, -4), ("version", 9, -2),
                              ("stride_node", 8, -5), ("temperature", 0.0, -6), ("levels", 0, -3),
                              ("flags", 8, -3), ("flags", 3, -3)]:
         dd, _ = binding._desc(x, sh.Tree.heap(3), 1.0)
