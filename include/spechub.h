@@ -217,6 +217,37 @@ int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const v
                     const spechub_node_out *node_out, const spechub_seq_out *seq_out,
                     void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * SpecHub, RRS and RRSw side by side on the same p, q and uniforms (the
+ * comparison of Section 5: all methods verify the same draft tree shapes).
+ * Results are those of spechub_draft_sample / rrs_draft_sample(0) /
+ * rrs_draft_sample(1), bit for bit; index 0 = SpecHub, 1 = RRS, 2 = RRSw.
+ * Where the rows are bf16, 16-byte aligned, vocab % 8 == 0 and vocab >= 8192,
+ * one kernel reads q once for the three methods (x1 is the same draw for all,
+ * since they share u_d1); otherwise the three calls are made one after another.
+ * desc->k must be 2.  draft_tokens[m] is [B][N][2] (out, required);
+ * status may be NULL or hold three pointers, each of which may be NULL;
+ * hub and draft_prob are SpecHub's.
+ */
+int mdsd_compare_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                              int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
+                              uint32_t *const status[3], void *stream);
+
+/*
+ * Verification by the three methods from shared reads of p and q, then one tree
+ * walk per method.  node_out[m] (three records, accept_idx and token required
+ * in each) and seq_out (NULL, or three records) receive what
+ * spechub_verify_tree / rrs_verify_tree(0) / rrs_verify_tree(1) would write,
+ * bit for bit, given draft_tokens[m] ([B][N][2], in) and the same uniforms.
+ * On the shapes named above one kernel makes three passes over a row pair
+ * (common max / sum / hub; S1, S2, R, A1 and RRSw's renormaliser; the two
+ * second-stage residual masses of Algorithm 1) instead of eight.
+ */
+int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                             const int32_t *const draft_tokens[3], const float *uniforms,
+                             const spechub_node_out node_out[3], const spechub_seq_out *seq_out,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
 /* Scratch bytes the two verify calls need for this descriptor (0 is possible). */
 size_t spechub_workspace_bytes(const spechub_desc *desc);
 

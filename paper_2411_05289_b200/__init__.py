@@ -14,6 +14,8 @@ from .binding import (  # noqa: F401
     abi_version,
     library_path,
     load_library,
+    mdsd_compare_draft_sample,
+    mdsd_compare_verify_tree,
     rrs_draft_sample,
     rrs_verify_tree,
     set_row_split,

@@ -95,6 +95,13 @@ def load_library(build_if_missing: bool = True):
     lib.rrs_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, i32,
                                     ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
                                     ctypes.c_size_t, vp]
+    lib.mdsd_compare_draft_sample.restype = i32
+    lib.mdsd_compare_draft_sample.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp, vp,
+                                              ctypes.POINTER(vp), vp]
+    lib.mdsd_compare_verify_tree.restype = i32
+    lib.mdsd_compare_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp,
+                                             ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                             ctypes.c_size_t, vp]
     lib.spechub_workspace_bytes.restype = ctypes.c_size_t
     lib.spechub_workspace_bytes.argtypes = [ctypes.POINTER(_Desc)]
     lib.spechub_status_string.restype = ctypes.c_char_p
@@ -332,6 +339,63 @@ def rrs_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: T
     """RRS / RRSw verification of every node and the tree walk."""
     return _verify("rrsw" if without_replacement else "rrs", target_logits, draft_logits, draft_tokens,
                    uniforms, tree, temperature, stream, out, probabilities)
+
+
+METHODS = ("spechub", "rrs", "rrsw")
+
+
+def mdsd_compare_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
+    """Draft step of SpecHub, RRS and RRSw on the same q and uniforms.  Returns a dict keyed by
+    method name; each entry is what the method's own draft call returns."""
+    lib = load_library()
+    _need_k2(tree)
+    d, keep = _desc(draft_logits, tree, temperature)
+    B, N, _ = draft_logits.shape
+    dev = draft_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    tokens = [torch.empty((B, N, 2), dtype=torch.int32, device=dev) for _ in METHODS]
+    status = [torch.empty((B, N), dtype=torch.int32, device=dev) for _ in METHODS]
+    hub = torch.empty((B, N), dtype=torch.int32, device=dev)
+    prob = torch.empty((B, N, 2), dtype=torch.float32, device=dev)
+    tp = (ctypes.c_void_p * 3)(*[t.data_ptr() for t in tokens])
+    sp = (ctypes.c_void_p * 3)(*[t.data_ptr() for t in status])
+    _check(lib.mdsd_compare_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), tp, _ptr(hub),
+                                         _ptr(prob), sp, _stream_ptr(stream)))
+    return dict(spechub=dict(tokens=tokens[0], hub=hub, prob=prob, status=status[0]),
+                rrs=dict(tokens=tokens[1], status=status[1]),
+                rrsw=dict(tokens=tokens[2], status=status[2]))
+
+
+def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
+                             temperature=1.0, stream=None, out=None, probabilities=True):
+    """Verification and tree walk by SpecHub, RRS and RRSw from shared reads of p and q.
+    ``draft_tokens`` and ``out`` are dicts keyed by method name (``out`` entries as made by
+    ``alloc_verify_outputs``).  Returns ``out``."""
+    lib = load_library()
+    _need_k2(tree)
+    _same_layout(target_logits, draft_logits)
+    d, keep = _desc(target_logits, tree, temperature)
+    B, N, _ = target_logits.shape
+    dev = target_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    for m in METHODS:
+        t = draft_tokens[m]
+        if t.dtype != torch.int32 or tuple(t.shape) != (B, N, 2) or not t.is_contiguous() or t.device != dev:
+            raise ValueError("draft_tokens[%s] must be a contiguous int32 [batch][nodes][2] tensor" % m)
+    if out is None:
+        out = {m: alloc_verify_outputs(B, N, tree.levels, dev) for m in METHODS}
+    no = (_NodeOut * 3)(*[
+        _NodeOut(*[out[m][k].data_ptr() if (probabilities or k not in ("beta", "rate")) else None
+                   for k in ("accept_idx", "token", "hub", "beta", "rate", "status")]) for m in METHODS])
+    so = (_SeqOut * 3)(*[
+        _SeqOut(*[out[m][k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])
+        for m in METHODS])
+    tp = (ctypes.c_void_p * 3)(*[draft_tokens[m].data_ptr() for m in METHODS])
+    ws_bytes = lib.spechub_workspace_bytes(ctypes.byref(d))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
+    _check(lib.mdsd_compare_verify_tree(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), tp,
+                                        _ptr(uniforms), no, so, _ptr(ws), ws_bytes, _stream_ptr(stream)))
+    return out
 
 
 def workspace_bytes(logits, tree: Tree, temperature=1.0) -> int:

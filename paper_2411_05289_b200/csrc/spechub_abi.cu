@@ -9,6 +9,7 @@
 #include "spechub_stream.cuh"
 #include "spechub_lean.cuh"
 #include "spechub_kary.cuh"
+#include "spechub_fused.cuh"
 
 namespace {
 
@@ -168,6 +169,30 @@ void launch_verify(const spechub_desc *d, const RowArgs &a, bool al, unsigned ro
     }
 }
 
+int launch_walk(const spechub_desc *d, const spechub_node_out *no, const spechub_seq_out *so, cudaStream_t s) {
+    if (!(so && (so->n_accepted || so->n_emitted || so->path_nodes || so->path_tokens))) return SPECHUB_OK;
+    WalkArgs w;
+    w.accept_idx = no->accept_idx;
+    w.token = no->token;
+    w.child = d->child;
+    w.node_kind = d->node_kind;
+    w.n_accepted = so->n_accepted;
+    w.n_emitted = so->n_emitted;
+    w.path_nodes = so->path_nodes;
+    w.path_tokens = so->path_tokens;
+    w.batch = d->batch;
+    w.nodes = d->nodes;
+    w.levels = d->levels;
+    if (d->k > 2) {
+        WalkKArgs wk;
+        wk.w = w; wk.k = d->k;
+        walk_k_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(wk);
+    } else {
+        walk_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(w);
+    }
+    return launch_status();
+}
+
 int verify_common(const spechub_desc *d, const void *target_logits, const void *draft_logits,
                   const int32_t *draft_tokens, const float *uniforms, int method,
                   const spechub_node_out *no, const spechub_seq_out *so, void *workspace,
@@ -212,30 +237,78 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
     } else if (method == kSpecHub) launch_verify<kSpecHub>(d, a, al, rows, th, s);
     else if (method == kRRS) launch_verify<kRRS>(d, a, al, rows, th, s);
     else launch_verify<kRRSw>(d, a, al, rows, th, s);
-    int lrc = launch_status();
+    const int lrc = launch_status();
     if (lrc != SPECHUB_OK) return lrc;
-    if (so && (so->n_accepted || so->n_emitted || so->path_nodes || so->path_tokens)) {
-        WalkArgs w;
-        w.accept_idx = no->accept_idx;
-        w.token = no->token;
-        w.child = d->child;
-        w.node_kind = d->node_kind;
-        w.n_accepted = so->n_accepted;
-        w.n_emitted = so->n_emitted;
-        w.path_nodes = so->path_nodes;
-        w.path_tokens = so->path_tokens;
-        w.batch = d->batch;
-        w.nodes = d->nodes;
-        w.levels = d->levels;
-        if (d->k > 2) {
-            WalkKArgs wk;
-            wk.w = w; wk.k = d->k;
-            walk_k_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(wk);
-        } else {
-            walk_kernel<<<(d->batch + 127) / 128, 128, 0, s>>>(w);
+    return launch_walk(d, no, so, s);
+}
+
+// One kernel for the three methods where the lean kernels apply, the three separate paths otherwise.
+int compare_draft(const spechub_desc *d, const void *draft_logits, const float *uniforms,
+                  int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
+                  uint32_t *const status[3], void *stream) {
+    const int rc = check_desc(d);
+    if (rc != SPECHUB_OK) return rc;
+    if (d->k != 2) return SPECHUB_ERR_SHAPE;
+    if (d->batch == 0) return SPECHUB_OK;
+    if (!draft_logits || !uniforms || !draft_tokens || !draft_tokens[0] || !draft_tokens[1] || !draft_tokens[2])
+        return SPECHUB_ERR_NULL;
+    if (!lean_ok(d, rows_aligned(d, draft_logits))) {
+        for (int m = 0; m < 3; ++m) {
+            const int mrc = draft_common(d, draft_logits, uniforms, m, draft_tokens[m], m == 0 ? hub : nullptr,
+                                         m == 0 ? draft_prob : nullptr, status ? status[m] : nullptr, stream);
+            if (mrc != SPECHUB_OK) return mrc;
         }
-        lrc = launch_status();
+        return SPECHUB_OK;
     }
+    FusedArgs f = {};
+    f.r = base_args(d);
+    f.r.draft = draft_logits;
+    f.r.uniforms = uniforms;
+    for (int m = 0; m < 3; ++m) {
+        f.tok_out[m] = draft_tokens[m];
+        f.dstatus[m] = status ? status[m] : nullptr;
+    }
+    const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
+    fused_draft_kernel<kLeanThreads><<<rows, kLeanThreads, 0, static_cast<cudaStream_t>(stream)>>>(f, hub, draft_prob);
+    return launch_status();
+}
+
+int compare_verify(const spechub_desc *d, const void *target_logits, const void *draft_logits,
+                   const int32_t *const draft_tokens[3], const float *uniforms,
+                   const spechub_node_out *no, const spechub_seq_out *so, void *workspace,
+                   size_t workspace_bytes, void *stream) {
+    const int rc = check_desc(d);
+    if (rc != SPECHUB_OK) return rc;
+    if (d->k != 2) return SPECHUB_ERR_SHAPE;
+    if (d->batch == 0) return SPECHUB_OK;
+    if (!target_logits || !draft_logits || !uniforms || !no || !draft_tokens) return SPECHUB_ERR_NULL;
+    for (int m = 0; m < 3; ++m)
+        if (!draft_tokens[m] || !no[m].accept_idx || !no[m].token) return SPECHUB_ERR_NULL;
+    if (workspace_bytes < spechub_workspace_bytes(d)) return SPECHUB_ERR_WORKSPACE;
+    const bool al = rows_aligned(d, target_logits) && rows_aligned(d, draft_logits);
+    if (!lean_ok(d, al)) {
+        for (int m = 0; m < 3; ++m) {
+            const int mrc = verify_common(d, target_logits, draft_logits, draft_tokens[m], uniforms, m, &no[m],
+                                          so ? &so[m] : nullptr, workspace, workspace_bytes, stream);
+            if (mrc != SPECHUB_OK) return mrc;
+        }
+        return SPECHUB_OK;
+    }
+    FusedArgs f = {};
+    f.r = base_args(d);
+    f.r.target = target_logits;
+    f.r.draft = draft_logits;
+    f.r.uniforms = uniforms;
+    for (int m = 0; m < 3; ++m) {
+        f.tok[m] = draft_tokens[m];
+        f.out[m].accept_idx = no[m].accept_idx; f.out[m].token = no[m].token; f.out[m].hub = no[m].hub;
+        f.out[m].beta = no[m].beta; f.out[m].rate = no[m].rate; f.out[m].status = no[m].status;
+    }
+    const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
+    int lrc = launch_status();
+    for (int m = 0; m < 3 && lrc == SPECHUB_OK && so; ++m) lrc = launch_walk(d, &no[m], &so[m], s);
     return lrc;
 }
 
@@ -274,6 +347,20 @@ int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const v
     return verify_common(desc, target_logits, draft_logits, draft_tokens, uniforms,
                          without_replacement ? kRRSw : kRRS, node_out, seq_out, workspace,
                          workspace_bytes, stream);
+}
+
+int mdsd_compare_draft_sample(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                              int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
+                              uint32_t *const status[3], void *stream) {
+    return compare_draft(desc, draft_logits, uniforms, draft_tokens, hub, draft_prob, status, stream);
+}
+
+int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                             const int32_t *const draft_tokens[3], const float *uniforms,
+                             const spechub_node_out node_out[3], const spechub_seq_out *seq_out,
+                             void *workspace, size_t workspace_bytes, void *stream) {
+    return compare_verify(desc, target_logits, draft_logits, draft_tokens, uniforms, node_out, seq_out,
+                          workspace, workspace_bytes, stream);
 }
 
 size_t spechub_workspace_bytes(const spechub_desc *desc) {

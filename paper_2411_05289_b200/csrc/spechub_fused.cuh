@@ -1,0 +1,390 @@
+// SpecHub, RRS and RRSw on the same rows in one kernel (large-vocabulary bf16 shapes).
+//
+// The three methods read the same p and q.  Pass A (max, sum of exponentials, hub) is common to
+// them; one pass B forms p(y), q(y) once and feeds SpecHub's transport sums, RRS's A1 and RRSw's
+// renormaliser; one pass C gives the two second-stage residual masses.  Three passes over a row
+// pair instead of 2 + 3 + 3, 6 ex2 per vocabulary pair instead of 16.  Every sum is accumulated
+// exactly as in lean_verify_kernel / lean_draft_kernel, so the results are bit-identical to the
+// separate calls.
+#pragma once
+
+#include "spechub.h"
+#include "spechub_common.cuh"
+#include "spechub_stream.cuh"
+#include "spechub_lean.cuh"
+
+namespace spechub {
+
+struct NodeOutPtrs {
+    int32_t *accept_idx, *token, *hub;
+    float *beta, *rate;
+    uint32_t *status;
+};
+struct FusedArgs {
+    RowArgs r;                 // target, draft, uniforms, temperature, node_kind, shape
+    const int32_t *tok[3];     // draft tokens of SpecHub, RRS, RRSw (verify)
+    int32_t *tok_out[3];       // (draft)
+    NodeOutPtrs out[3];
+    uint32_t *dstatus[3];      // draft status
+};
+
+__device__ __forceinline__ void write_node3(const NodeOutPtrs &p, long long r, const NodeResult &o, bool tok_elsewhere) {
+    p.accept_idx[r] = o.accept_idx;
+    if (!tok_elsewhere) p.token[r] = o.token;
+    if (p.hub) p.hub[r] = o.hub;
+    if (p.beta) { p.beta[2 * r] = o.beta[0]; p.beta[2 * r + 1] = o.beta[1]; }
+    if (p.rate) { p.rate[3 * r] = o.rate[0]; p.rate[3 * r + 1] = o.rate[1]; p.rate[3 * r + 2] = o.rate[2]; }
+    if (p.status) p.status[r] = o.status;
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(FusedArgs A) {
+    __shared__ LeanShared sh;
+    const RowArgs &a = A.r;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    const __nv_bfloat16 *rowp = static_cast<const __nv_bfloat16 *>(a.target) + b * a.stride_seq + n * a.stride_node;
+    const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(rowp), *vq = reinterpret_cast<const uint4 *>(rowq);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const int last_vi = (lo + lane < hi) ? lo + lane + ((hi - 1 - lo - lane) / 32) * 32 : lo - 1;
+    const float k = kLog2e / temperature_of(a, b);
+    const float r1 = a.uniforms[r * 5 + 2], r2 = a.uniforms[r * 5 + 3], ures = a.uniforms[r * 5 + 4];
+    const float pinf = -neg_inf();
+    const bool leaf = a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF;
+    const bool t0 = threadIdx.x == 0;
+
+    NodeResult o[3];
+    bool elsewhere[3] = {false, false, false};
+#pragma unroll
+    for (int m = 0; m < 3; ++m) {
+        o[m].accept_idx = -1; o[m].token = -1; o[m].hub = -1; o[m].status = 0;
+        o[m].beta[0] = o[m].beta[1] = 0.f; o[m].rate[0] = o[m].rate[1] = o[m].rate[2] = 0.f;
+    }
+    auto finish = [&]() {
+        if (!t0) return;
+#pragma unroll
+        for (int m = 0; m < 3; ++m) write_node3(A.out[m], r, o[m], elsewhere[m]);
+    };
+
+    LeanAcc tp, tq;
+    if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
+    else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
+    {
+        ArgMaxSum Ps, Qs;
+        if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        if (t0) {
+            sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
+            sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+        }
+    }
+    __syncthreads();
+    RowStat P, Q;
+    merge_slices<1>(sh, 0, k, P);
+    merge_slices<1>(sh, 1, k, Q);
+    const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
+    const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
+    auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
+    auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
+    auto draw_from_p = [&]() { return lean_sample_row<1>(g, rowp, k, P, 0, -1, ures, 0, sh); };
+
+    if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
+        for (int m = 0; m < 3; ++m) o[m].status = SPECHUB_ST_NONFINITE;
+        finish();
+        return;
+    }
+    if (leaf) {
+        const int tok = draw_from_p();   // the three methods share u_res, so they share the bonus token
+        for (int m = 0; m < 3; ++m) { o[m].token = tok; o[m].rate[2] = 1.f; }
+        finish();
+        return;
+    }
+    if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) {
+        for (int m = 0; m < 3; ++m) o[m].status = SPECHUB_ST_NONFINITE;
+        finish();
+        return;
+    }
+    // ---- per-method draft tokens ----
+    const int hubtok = Q.idx;
+    const int sx1 = A.tok[0][2 * r], sx2 = A.tok[0][2 * r + 1];
+    const bool pair_xa = (sx2 == hubtok && sx1 != hubtok), pair_ax = (sx1 == hubtok && sx2 != hubtok);
+    const int x = pair_xa ? sx1 : sx2;
+    const bool ok_s = (pair_xa || pair_ax) && x >= 0 && x < a.vocab;
+    int rx1[2], rx2[2];
+    bool ok_r[2];
+    for (int m = 0; m < 2; ++m) {
+        rx1[m] = A.tok[1 + m][2 * r]; rx2[m] = A.tok[1 + m][2 * r + 1];
+        ok_r[m] = rx1[m] >= 0 && rx1[m] < a.vocab && rx2[m] >= 0 && rx2[m] < a.vocab;
+    }
+    o[0].hub = hubtok;
+    if (!ok_s) o[0].status = SPECHUB_ST_TOKEN_RANGE;
+    if (!ok_r[0]) o[1].status = SPECHUB_ST_TOKEN_RANGE;
+    if (!ok_r[1]) o[2].status = SPECHUB_ST_TOKEN_RANGE;
+    const bool degenerate = !(Q.sx > 0.f);
+    const float c = degenerate ? 0.f : 1.f / Q.sx;
+    const float qa = invZq, rest = Q.sx * invZq;
+    const int hubvec = hubtok >> 3, hubel = hubtok & 7;
+    const int wx1 = ok_r[1] ? rx1[1] : -1;            // RRSw's first draft (left out of its renormaliser)
+    const int wvec = wx1 >> 3, wel = wx1 & 7;
+
+    // ---- pass B (backwards): SpecHub S1, S2, R; A1; RRSw's sum of q outside its x1 ----
+    float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
+    float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
+#pragma unroll 2
+    for (int vi = last_vi; vi >= lo; vi -= 32) {
+        float fp[8], fq[8];
+        unpack_bf16x8(vp[vi], fp);
+        unpack_bf16x8(vq[vi], fq);
+        float pp[8], qq[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
+            a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
+        }
+        {
+            float qw[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) qw[i] = qq[i];
+            if (vi == wvec) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i == wel) qw[i] = 0.f;
+            }
+            dna += (qw[0] + qw[1]) + (qw[2] + qw[3]);
+            dnb += (qw[4] + qw[5]) + (qw[6] + qw[7]);
+        }
+        if (vi == hubvec) {   // SpecHub's sums run over ids != a
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i == hubel) { pp[i] = 0.f; qq[i] = 0.f; }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            float d, t;
+            transport_terms(pp[i], qq[i], c, d, t);
+            s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
+            transport_terms(pp[i + 1], qq[i + 1], c, d, t);
+            s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
+        }
+    }
+    float accB[5] = {s1a + s1b, s2a + s2b, ra + rb, a1a + a1b, dna + dnb};
+    lean_block_sums<5, 0>(accB, sh);   // per-warp R stays in sh.acc[2]
+    const float S1 = accB[0], S2 = degenerate ? qa : accB[1], R = accB[2], A1 = accB[3], den = accB[4];
+
+    // ---- pass C (forwards): second-stage residual masses of RRS and RRSw ----
+    const bool q1_zero = !(den > 0.f);
+    const float A1g[2] = {A1, A1 * (q1_zero ? 0.f : 1.f / den)};
+    float w0a = 0.f, w0b = 0.f, w1a = 0.f, w1b = 0.f;
+#pragma unroll 2
+    for (int vi = lo + lane; vi < hi; vi += 32) {
+        float fp[8], fq[8];
+        unpack_bf16x8(vp[vi], fp);
+        unpack_bf16x8(vq[vi], fq);
+        float sc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sc[i] = A1g[1];
+        if (vi == wvec) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i == wel) sc[i] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            const float p0 = prob_of(fp[i], k, cP, invZp), q0 = prob_of(fq[i], k, cQ, invZq);
+            const float p1 = prob_of(fp[i + 1], k, cP, invZp), q1 = prob_of(fq[i + 1], k, cQ, invZq);
+            float d, t;
+            transport_terms(p0, q0, A1g[0], d, t); w0a += fmaxf(t, 0.f);
+            transport_terms(p1, q1, A1g[0], d, t); w0b += fmaxf(t, 0.f);
+            transport_terms(p0, q0, sc[i], d, t); w1a += fmaxf(t, 0.f);
+            transport_terms(p1, q1, sc[i + 1], d, t); w1b += fmaxf(t, 0.f);
+        }
+    }
+    float accC[2] = {w0a + w0b, w1a + w1b};
+    lean_block_sums<2, 5>(accC, sh);   // per-warp W2 stay in sh.acc[5], sh.acc[6]
+    __syncthreads();
+
+    // ---- SpecHub decisions (Algorithm 3) ----
+    if (ok_s) {
+        NodeResult &s = o[0];
+        const float pa = prob_p(hubtok);
+        const float hub_left = fmaxf(pa - S2, 0.f);
+        s.rate[0] = fmaxf(rest - S1, 0.f) + fminf(pa, S2);
+        s.rate[1] = (degenerate ? 0.f : fmaxf(qa - S2, 0.f)) + fminf(hub_left, S1);
+        s.rate[2] = R;
+        if (degenerate) s.status |= SPECHUB_ST_DEGENERATE_Q;
+        const float px = prob_p(x), qx = prob_q(x);
+        bool acc1, acc2;
+        if (pair_xa) {
+            acc1 = accept_test(r1, px, qx, s.beta[0], true, s.status);
+            if (acc1) { s.accept_idx = 0; s.token = x; }
+            acc2 = accept_test(r2, hub_left, S1, s.beta[1], !acc1, s.status);
+            if (!acc1 && acc2) { s.accept_idx = 1; s.token = hubtok; }
+        } else {
+            acc1 = accept_test(r1, fmaxf(__fsub_rn(px, qx), 0.f), c * qx, s.beta[0], true, s.status);
+            if (acc1) { s.accept_idx = 1; s.token = x; }
+            acc2 = accept_test(r2, pa, S2, s.beta[1], !acc1, s.status);
+            if (!acc1 && acc2) { s.accept_idx = 0; s.token = hubtok; }
+        }
+        if (!(acc1 || acc2)) {
+            s.accept_idx = -1;
+            int tok;
+            if (R > 0.f) {
+                if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
+                __syncthreads();
+                auto wf = [&](int vi, float(&w)[8]) {
+                    float fp[8], fq[8];
+                    unpack_bf16x8(vp[vi], fp);
+                    unpack_bf16x8(vq[vi], fq);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float d, t;
+                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                        w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
+                    }
+                };
+                tok = block_sample3(g, wf, sh, ures * R);
+            } else {
+                s.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                tok = draw_from_p();
+            }
+            s.token = tok;
+        }
+    }
+    // ---- RRS / RRSw decisions (Algorithm 1) ----
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+        if (!ok_r[m]) continue;
+        NodeResult &s = o[1 + m];
+        const bool wo = (m == 1);
+        const float W2 = accC[m];
+        const int x1 = rx1[m], x2 = rx2[m];
+        s.rate[0] = fmaxf(1.f - A1, 0.f);
+        s.rate[1] = fmaxf(A1 - W2, 0.f);
+        s.rate[2] = W2;
+        const float px1 = prob_p(x1), qx1 = prob_q(x1), px2 = prob_p(x2), qx2 = prob_q(x2);
+        const bool acc1 = accept_test(r1, px1, qx1, s.beta[0], true, s.status);
+        if (acc1) { s.accept_idx = 0; s.token = x1; }
+        if (!acc1 && wo && q1_zero) s.status |= SPECHUB_ST_DEGENERATE_Q;
+        bool acc2 = false;
+        if (A1 > 0.f) {
+            const float q1x2 = (wo && x2 == x1) ? 0.f : A1g[m] * qx2;
+            acc2 = accept_test(r2, fmaxf(__fsub_rn(px2, qx2), 0.f), q1x2, s.beta[1], !acc1, s.status);
+        }
+        if (!acc1 && acc2) { s.accept_idx = 1; s.token = x2; }
+        if (!(acc1 || acc2)) {
+            s.accept_idx = -1;
+            int tok;
+            if (A1 > 0.f && W2 > 0.f) {
+                if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[5 + m][threadIdx.x];
+                __syncthreads();
+                const float coef = A1g[m];
+                auto wf = [&](int vi, float(&w)[8]) {
+                    float fp[8], fq[8];
+                    unpack_bf16x8(vp[vi], fp);
+                    unpack_bf16x8(vq[vi], fq);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float d, t;
+                        const float sc = (wo && vi * 8 + i == x1) ? 0.f : coef;
+                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc, d, t);
+                        w[i] = fmaxf(t, 0.f);
+                    }
+                };
+                tok = block_sample3(g, wf, sh, ures * W2);
+            } else {
+                s.status |= SPECHUB_ST_ZERO_RESIDUAL;
+                tok = draw_from_p();
+            }
+            s.token = tok;
+        }
+    }
+    finish();
+}
+
+// Draft step of the three methods from one read of q.  x1 ~ q is the same draw for all three
+// (they share u_d1).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(FusedArgs A, int32_t *hub_out,
+                                                                            float *draft_prob) {
+    __shared__ LeanShared sh;
+    const RowArgs &a = A.r;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vq = reinterpret_cast<const uint4 *>(rowq);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const float k = kLog2e / temperature_of(a, b);
+    const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
+    const bool t0 = threadIdx.x == 0;
+
+    LeanAcc tq, unused;
+    lean_pass_a<false>(vq, vq, lo, hi, lane, k, tq, unused);
+    {
+        ArgMaxSum q, unusedq;
+        lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
+        if (t0) { sh.x_ml[0] = q.ml; sh.x_sx[0] = q.sx; sh.x_idx[0] = q.idx; }
+    }
+    __syncthreads();
+    RowStat Q;
+    merge_slices<1>(sh, 0, k, Q);
+    const float Zq = Q.sx + 1.f;
+    if (!(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf())) {
+        if (t0) {
+            for (int m = 0; m < 3; ++m) {
+                A.tok_out[m][2 * r] = -1; A.tok_out[m][2 * r + 1] = -1;
+                if (A.dstatus[m]) A.dstatus[m][r] = SPECHUB_ST_NONFINITE;
+            }
+            if (hub_out) hub_out[r] = -1;
+            if (draft_prob) { draft_prob[2 * r] = 0.f; draft_prob[2 * r + 1] = 0.f; }
+        }
+        return;
+    }
+    const int hubtok = Q.idx;
+    const int x1 = lean_sample_row<1>(g, rowq, k, Q, 0, -1, u1, 0, sh);
+    uint32_t st[3] = {0, 0, 0};
+    int x2[3];
+    // SpecHub (Section 4)
+    const float prob0 = 1.f / Zq;
+    float prob1 = 0.f;
+    if (x1 != hubtok) {
+        x2[0] = hubtok;
+        prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)) / Zq;
+    } else if (!(Q.sx > 0.f)) {
+        x2[0] = (hubtok == 0) ? 1 : 0;
+        st[0] |= SPECHUB_ST_DEGENERATE_Q;
+    } else {
+        x2[0] = lean_sample_row<1>(g, rowq, k, Q, 0, hubtok, u2, 0, sh);
+        prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2[0]), k, -Q.C)) / Q.sx;
+    }
+    // RRS: an independent second draw
+    x2[1] = lean_sample_row<1>(g, rowq, k, Q, 0, -1, u2, 0, sh);
+    // RRSw: q with q(x1) set to 0
+    {
+        float m0 = slice_mass<1>(sh, 0, Q, 0, x1, k);
+        if (sh.x_idx[0] != x1) m0 = fmaxf(m0 - ex2(__fmaf_rn(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)), 0.f);
+        if (m0 > 0.f) {
+            x2[2] = lean_sample_slice(g, rowq, k, Q, x1, u2 * m0, 0, sh);
+        } else {
+            st[2] |= SPECHUB_ST_DEGENERATE_Q;
+            x2[2] = (x1 == 0) ? 1 : 0;
+        }
+    }
+    if (t0) {
+        for (int m = 0; m < 3; ++m) {
+            A.tok_out[m][2 * r] = x1;
+            A.tok_out[m][2 * r + 1] = x2[m];
+            if (A.dstatus[m]) A.dstatus[m][r] = st[m];
+        }
+        if (hub_out) hub_out[r] = hubtok;
+        if (draft_prob) { draft_prob[2 * r] = prob0; draft_prob[2 * r + 1] = prob1; }
+    }
+}
+
+}  // namespace spechub

@@ -42,7 +42,7 @@ struct LeanShared {
     float wml[2][kLeanMaxWarps];    // per-warp max logit (0 target, 1 draft)
     float wmass[2][kLeanMaxWarps];  // per-warp sum of exponentials on the row's scale, argmax left out
     int cand[2];                    // lowest index attaining the row maximum
-    float acc[4][kLeanMaxWarps];
+    float acc[8][kLeanMaxWarps];
     float mass[kLeanMaxWarps];
     float part[1024];  // sampler: per-thread block sums of the selected warp range
     float tt2;
@@ -495,20 +495,21 @@ __device__ int lean_sample_row(const Geo &g, const __nv_bfloat16 *row, float k, 
     return lean_sample_slice(g, row, k, st, excl, u * total - base, r, sh);
 }
 
-template <int NACC>
+// CTA sums of NACC per-thread accumulators; the per-warp sums stay in sh.acc[OFF + i][w].
+template <int NACC, int OFF = 0>
 __device__ __forceinline__ void lean_block_sums(float (&x)[NACC], LeanShared &sh) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll
     for (int i = 0; i < NACC; ++i) {
         const float s = warp_sum(x[i]);
-        if (lane == 0) sh.acc[i][warp] = s;
+        if (lane == 0) sh.acc[OFF + i][warp] = s;
     }
     __syncthreads();
     const int nwarps = blockDim.x >> 5;
 #pragma unroll
     for (int i = 0; i < NACC; ++i) {
         float t = 0.f;
-        for (int w = 0; w < nwarps; ++w) t += sh.acc[i][w];
+        for (int w = 0; w < nwarps; ++w) t += sh.acc[OFF + i][w];
         x[i] = t;
     }
 }

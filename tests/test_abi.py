@@ -13,12 +13,13 @@ def declared_functions():
     src = open(os.path.join(ROOT, "include", "spechub.h")).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
     names = re.findall(r"\b([a-z_0-9]+)\s*\(", src)
-    return sorted(set(n for n in names if n.startswith(("spechub_", "rrs_"))))
+    return sorted(set(n for n in names if n.startswith(("spechub_", "rrs_", "mdsd_"))))
 
 
 def test_header_declares_the_expected_entry_points():
     assert declared_functions() == sorted([
         "spechub_draft_sample", "rrs_draft_sample", "spechub_verify_tree", "rrs_verify_tree",
+        "mdsd_compare_draft_sample", "mdsd_compare_verify_tree",
         "spechub_workspace_bytes", "spechub_status_string", "spechub_abi_version"])
 
 
