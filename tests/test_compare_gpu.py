@@ -105,8 +105,7 @@ def test_compare_calls(sh, V, dtype, paper):
 
 
 def test_compare_calls_reject_more_than_two_drafts(sh):
-    lp, lq, un = make_case(8192, "bf16", 3, B=1, N=4)
-    tq = workloads.to_device(lq, "bf16")
+    tq = torch.zeros((1, 4, 8192), dtype=torch.bfloat16, device="cuda")
     tree = sh.Tree.kary(3, 2)
     with pytest.raises(ValueError):
         sh.mdsd_compare_draft_sample(tq, torch.zeros((1, 4, 7), device="cuda"), tree, 1.0)
