@@ -305,6 +305,22 @@ def main():
     barrier()
     lite_ms = q0.elapsed_time(q1) / args.steps
 
+    # ---- extra: the same step through the three-method calls (shared reads of p and q) ----
+    def fused_step():
+        d = sh.mdsd_compare_draft_sample(tq, un, tree, cfg.temperature)
+        sh.mdsd_compare_verify_tree(tp, tq, {m: d[m]["tokens"] for m in METHODS}, un, tree, cfg.temperature,
+                                    out=outs)
+
+    for _ in range(3):
+        fused_step()
+    barrier()
+    q0.record(stream)
+    for _ in range(args.steps):
+        fused_step()
+    q1.record(stream)
+    barrier()
+    fused_ms = q0.elapsed_time(q1) / args.steps
+
     # ---- end to end: host buffers in, host results out, through the public API ----
     esz = 2 if cfg.dtype == "bf16" else 4
     h_tp = torch.empty(tp.shape, dtype=tp.dtype, pin_memory=True); h_tp.copy_(tp)
@@ -386,6 +402,11 @@ def main():
                     "ms_per_launch": lite_ms, "nodes_per_s": B * N / (lite_ms * 1e-3),
                     "note": "beta / rate not requested: rows whose first test accepts skip pass B; "
                             "not part of `value`"},
+                "step_through_three_method_calls": {
+                    "ms_per_step": fused_ms, "nodes_per_s": len(METHODS) * B * N / (fused_ms * 1e-3),
+                    "gpu_launches_per_step": 5,
+                    "note": "mdsd_compare_draft_sample + mdsd_compare_verify_tree: same outputs as the "
+                            "nine launches of the timed step, bit for bit; this rank only; not part of `value`"},
             },
         }
         sfp = line["special_function_pipe"]
