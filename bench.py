@@ -365,7 +365,7 @@ def main():
 
     # The batch goes through in chunks of whole sequences on two streams, so that the copy of one
     # chunk overlaps the kernels of the one before; the library only enqueues on the given stream.
-    n_chunks = min(8, B)
+    n_chunks = max(1, min(8, B, int(input_bytes(cfg) // 400e6)))  # chunks of >= 0.4 GB: launches stay rare
     bounds = [(B * i // n_chunks, B * (i + 1) // n_chunks) for i in range(n_chunks)]
     side = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
     chunk_outs = [{m: {k: v[b0:b1] for k, v in outs[m].items()} for m in METHODS} for b0, b1 in bounds]
