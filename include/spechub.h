@@ -248,6 +248,59 @@ int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits
                              const spechub_node_out node_out[3], const spechub_seq_out *seq_out,
                              void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Tree walk alone (Figure 2) over per-node results already in device memory:
+ * accept_idx, token [B][N] (in), seq_out as in spechub_verify_tree.  Used after
+ * the vocabulary-sharded phases below, once the tokens have been exchanged.
+ */
+int spechub_walk_tree(const spechub_desc *desc, const int32_t *accept_idx, const int32_t *token,
+                      const spechub_seq_out *seq_out, void *stream);
+
+/*
+ * SpecHub with the vocabulary axis sharded over ranks (each rank's LM head
+ * produces the logits of a contiguous id range).  The paper has no counterpart:
+ * it states the method on whole distributions (Section 4, Algorithm 3); these
+ * calls compute the same quantities from slices.  desc->vocab is the width of
+ * this rank's slice, the logits pointers are its slices ([B][N][vocab] with the
+ * descriptor's strides); token ids everywhere are global.  desc->k must be 2.
+ *
+ * The caller runs, per rank and in lockstep:
+ *   draft:  spechub_shard_stats(target = NULL) -> all-gather of stats in rank
+ *           order -> spechub_shard_draft -> element-wise maximum of cand over
+ *           ranks -> spechub_shard_draft_finish;
+ *   verify: spechub_shard_stats -> all-gather -> spechub_shard_sums ->
+ *           all-gather -> spechub_shard_decide -> element-wise maximum of
+ *           node_out->token over ranks -> spechub_walk_tree.
+ * stats, sums: [B][N][8] floats (out); gathered_*: [nranks][B][N][8] (in).
+ * All ranks take identical decisions (the gathered partials are merged in rank
+ * order everywhere); a residual or bonus token is drawn by the rank whose slice
+ * holds the inverse-CDF target and is -2 on the others until the maximum is
+ * taken.  Results agree with spechub_draft_sample / spechub_verify_tree on the
+ * concatenated rows up to fp32 summation order.
+ */
+typedef struct {
+    int32_t rank, nranks;     /* 0 <= rank < nranks <= 64 */
+    int32_t id_offset;        /* global id of this slice's first token */
+    int32_t vocab_total;      /* sum of the slices' widths */
+} spechub_shard;
+
+int spechub_shard_stats(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                        const void *draft_slice, float *stats, void *stream);
+int spechub_shard_sums(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                       const void *draft_slice, const int32_t *draft_tokens, const float *gathered_stats,
+                       float *sums, void *stream);
+int spechub_shard_decide(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                         const void *draft_slice, const int32_t *draft_tokens, const float *uniforms,
+                         const float *gathered_stats, const float *gathered_sums,
+                         const spechub_node_out *node_out, void *stream);
+/* cand [B][N][2] (out): x1 and the second draw of a pair (a, x); -2 where another rank draws. */
+int spechub_shard_draft(const spechub_desc *desc, const spechub_shard *shard, const void *draft_slice,
+                        const float *uniforms, const float *gathered_stats, int32_t *cand, void *stream);
+/* cand_max: cand after the maximum over ranks; draft_tokens [B][N][2], hub, status as in spechub_draft_sample. */
+int spechub_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard,
+                               const float *gathered_stats, const int32_t *cand_max,
+                               int32_t *draft_tokens, int32_t *hub, uint32_t *status, void *stream);
+
 /* Scratch bytes the two verify calls need for this descriptor (0 is possible). */
 size_t spechub_workspace_bytes(const spechub_desc *desc);
 

@@ -10,6 +10,7 @@
 #include "spechub_lean.cuh"
 #include "spechub_kary.cuh"
 #include "spechub_fused.cuh"
+#include "spechub_shard.cuh"
 
 namespace {
 
@@ -312,6 +313,51 @@ int compare_verify(const spechub_desc *d, const void *target_logits, const void 
     return lrc;
 }
 
+// ---- vocabulary-sharded phases ------------------------------------------------------------------
+int check_shard(const spechub_desc *d, const spechub_shard *sh) {
+    const int rc = check_desc(d);
+    if (rc != SPECHUB_OK) return rc;
+    if (!sh) return SPECHUB_ERR_NULL;
+    if (d->k != 2) return SPECHUB_ERR_SHAPE;
+    if (sh->nranks < 1 || sh->nranks > 64 || sh->rank < 0 || sh->rank >= sh->nranks || sh->id_offset < 0 ||
+        sh->vocab_total < 2 || (int64_t)sh->id_offset + d->vocab > sh->vocab_total)
+        return SPECHUB_ERR_SHAPE;
+    return SPECHUB_OK;
+}
+
+ShardArgs shard_args(const spechub_desc *d, const spechub_shard *sh) {
+    ShardArgs a = {};
+    a.r = base_args(d);
+    a.rank = sh->rank; a.nranks = sh->nranks; a.id_offset = sh->id_offset; a.vocab_total = sh->vocab_total;
+    a.rows = d->batch * (int64_t)d->nodes;
+    return a;
+}
+
+enum ShardPhase { kPhaseStats, kPhaseSums, kPhaseDecide, kPhaseDraft };
+
+template <typename LT, bool AL>
+void launch_shard_phase(int phase, const ShardArgs &a, unsigned rows, int th, cudaStream_t s) {
+    if (phase == kPhaseStats) shard_stats_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else if (phase == kPhaseSums) shard_sums_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else if (phase == kPhaseDecide) shard_decide_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else shard_draft_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+}
+
+int run_shard_phase(int phase, const spechub_desc *d, const ShardArgs &a, void *stream) {
+    const unsigned rows = (unsigned)a.rows;
+    const int th = threads_for(d);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool al = (!a.r.target || rows_aligned(d, a.r.target)) && (!a.r.draft || rows_aligned(d, a.r.draft));
+    if (d->dtype == SPECHUB_BF16) {
+        if (al) launch_shard_phase<__nv_bfloat16, true>(phase, a, rows, th, s);
+        else launch_shard_phase<__nv_bfloat16, false>(phase, a, rows, th, s);
+    } else {
+        if (al) launch_shard_phase<float, true>(phase, a, rows, th, s);
+        else launch_shard_phase<float, false>(phase, a, rows, th, s);
+    }
+    return launch_status();
+}
+
 }  // namespace
 
 extern "C" {
@@ -361,6 +407,85 @@ int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits
                              void *workspace, size_t workspace_bytes, void *stream) {
     return compare_verify(desc, target_logits, draft_logits, draft_tokens, uniforms, node_out, seq_out,
                           workspace, workspace_bytes, stream);
+}
+
+int spechub_walk_tree(const spechub_desc *desc, const int32_t *accept_idx, const int32_t *token,
+                      const spechub_seq_out *seq_out, void *stream) {
+    const int rc = check_desc(desc);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!accept_idx || !token || !seq_out) return SPECHUB_ERR_NULL;
+    spechub_node_out no = {};
+    no.accept_idx = const_cast<int32_t *>(accept_idx);
+    no.token = const_cast<int32_t *>(token);
+    return launch_walk(desc, &no, seq_out, static_cast<cudaStream_t>(stream));
+}
+
+int spechub_shard_stats(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                        const void *draft_slice, float *stats, void *stream) {
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!draft_slice || !stats) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.r.target = target_slice; a.r.draft = draft_slice; a.out = stats;
+    return run_shard_phase(kPhaseStats, desc, a, stream);
+}
+
+int spechub_shard_sums(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                       const void *draft_slice, const int32_t *draft_tokens, const float *gathered_stats,
+                       float *sums, void *stream) {
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!target_slice || !draft_slice || !draft_tokens || !gathered_stats || !sums) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.r.target = target_slice; a.r.draft = draft_slice; a.r.draft_tokens_in = draft_tokens;
+    a.gstats = gathered_stats; a.out = sums;
+    return run_shard_phase(kPhaseSums, desc, a, stream);
+}
+
+int spechub_shard_decide(const spechub_desc *desc, const spechub_shard *shard, const void *target_slice,
+                         const void *draft_slice, const int32_t *draft_tokens, const float *uniforms,
+                         const float *gathered_stats, const float *gathered_sums,
+                         const spechub_node_out *no, void *stream) {
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!target_slice || !draft_slice || !draft_tokens || !uniforms || !gathered_stats || !gathered_sums ||
+        !no || !no->accept_idx || !no->token)
+        return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.r.target = target_slice; a.r.draft = draft_slice; a.r.draft_tokens_in = draft_tokens;
+    a.r.uniforms = uniforms; a.gstats = gathered_stats; a.gsums = gathered_sums;
+    a.r.hub = no->hub; a.r.accept_idx = no->accept_idx; a.r.token = no->token;
+    a.r.beta = no->beta; a.r.rate = no->rate; a.r.status = no->status;
+    return run_shard_phase(kPhaseDecide, desc, a, stream);
+}
+
+int spechub_shard_draft(const spechub_desc *desc, const spechub_shard *shard, const void *draft_slice,
+                        const float *uniforms, const float *gathered_stats, int32_t *cand, void *stream) {
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!draft_slice || !uniforms || !gathered_stats || !cand) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.r.draft = draft_slice; a.r.uniforms = uniforms; a.gstats = gathered_stats; a.cand_out = cand;
+    return run_shard_phase(kPhaseDraft, desc, a, stream);
+}
+
+int spechub_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard,
+                               const float *gathered_stats, const int32_t *cand_max,
+                               int32_t *draft_tokens, int32_t *hub, uint32_t *status, void *stream) {
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!gathered_stats || !cand_max || !draft_tokens) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.gstats = gathered_stats; a.cand = cand_max;
+    a.r.draft_tokens_out = draft_tokens; a.r.hub = hub; a.r.status = status;
+    shard_draft_finish_kernel<<<(unsigned)((a.rows + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    return launch_status();
 }
 
 size_t spechub_workspace_bytes(const spechub_desc *desc) {

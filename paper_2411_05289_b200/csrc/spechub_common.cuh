@@ -235,13 +235,11 @@ __device__ __forceinline__ float warp_sum(float x) {
 // the lowest id whose inclusive prefix exceeds u * total; when rounding leaves
 // none inside the selected range, the last id with positive weight there; -1 when
 // the total is 0.  Must be called by all threads of the CTA.
+// block_sample_at takes the target prefix t itself (a draw whose total spans more than this CTA's
+// range); block_sample draws with u * (this range's total).
 template <int VW, class WF>
-__device__ int block_sample(const Geo &g, WF weights, const float *mass, float u, int *sh_tok) {
+__device__ int block_sample_at(const Geo &g, WF weights, const float *mass, float t, int *sh_tok) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float total = 0.f;
-    for (int w = 0; w < g.nwarps; ++w) total += mass[w];
-    if (!(total > 0.f)) return -1;
-    const float t = u * total;
     int wsel = -1, lastw = -1;
     float base = 0.f, lastbase = 0.f, run = 0.f;
     for (int w = 0; w < g.nwarps; ++w) {
@@ -253,6 +251,7 @@ __device__ int block_sample(const Geo &g, WF weights, const float *mass, float u
         }
         run += m;
     }
+    if (lastw < 0) return -1;
     if (wsel < 0) { wsel = lastw; base = lastbase; }
     if (warp == wsel) {
         const float tt = t - base;
@@ -314,6 +313,14 @@ __device__ int block_sample(const Geo &g, WF weights, const float *mass, float u
     const int tok = *sh_tok;
     __syncthreads();
     return tok;
+}
+
+template <int VW, class WF>
+__device__ int block_sample(const Geo &g, WF weights, const float *mass, float u, int *sh_tok) {
+    float total = 0.f;
+    for (int w = 0; w < g.nwarps; ++w) total += mass[w];
+    if (!(total > 0.f)) return -1;
+    return block_sample_at<VW>(g, weights, mass, u * total, sh_tok);
 }
 
 }  // namespace spechub

@@ -19,7 +19,9 @@ def declared_functions():
 def test_header_declares_the_expected_entry_points():
     assert declared_functions() == sorted([
         "spechub_draft_sample", "rrs_draft_sample", "spechub_verify_tree", "rrs_verify_tree",
-        "mdsd_compare_draft_sample", "mdsd_compare_verify_tree",
+        "mdsd_compare_draft_sample", "mdsd_compare_verify_tree", "spechub_walk_tree",
+        "spechub_shard_stats", "spechub_shard_sums", "spechub_shard_decide", "spechub_shard_draft",
+        "spechub_shard_draft_finish",
         "spechub_workspace_bytes", "spechub_status_string", "spechub_abi_version"])
 
 

@@ -1,0 +1,128 @@
+"""Vocabulary-sharded SpecHub: the ranks' phases run in lockstep on one GPU (the exchanges become a
+stack and an element-wise maximum), and the result is compared with the CPU oracle on the whole
+rows.  No kernel waits on another: each phase is an ordinary launch."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+import oracle  # noqa: E402
+import workloads  # noqa: E402
+import parity  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def sh():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2411_05289_b200 as lib
+
+    lib.load_library()
+    return lib
+
+
+def make_case(V, dtype, seed, B=4, N=7):
+    rng = np.random.default_rng(seed)
+    lp = rng.normal(0, 2.0, (B, N, V)).astype(np.float32)
+    lq = lp + rng.normal(0, 1.0, (B, N, V)).astype(np.float32)
+    lq[0, 1] = lp[0, 1]                                    # p = q
+    lq[1, 2] = -np.inf; lq[1, 2, V - 1] = 0.0              # one-hot q on the last rank
+    lq[2, 0] = -60.0; lq[2, 0, V // 2] = 0.0               # nearly one-hot q
+    lp[3, 3, : V // 2] = -np.inf; lq[3, 3, V // 2:] = -np.inf   # disjoint supports: whole slices empty
+    lp[1, 4] = np.round(lp[1, 4] * 2) / 2; lq[1, 4] = np.round(lq[1, 4] * 2) / 2   # ties across ranks
+    lq[0, 5, 7] = lq[0, 5].max() + 9.0                     # peaked draft
+    lp[2, 6, 3] = np.nan                                   # flagged target row
+    lq[3, 6, V - 2] = np.inf                               # flagged draft row
+    lp, lq = workloads.round_to_storage(lp, dtype), workloads.round_to_storage(lq, dtype)
+    un = rng.integers(0, 1 << 24, (B, N, 5)).astype(np.float32) * np.float32(2.0 ** -24)
+    return lp, lq, un
+
+
+def lockstep_draft(vs, slices_q, und, tree, shards, T):
+    ranks = [vs.ShardedDraft(q, und, tree, s, T) for q, (s, _) in zip(slices_q, shards)]
+    g = torch.stack([r.stats() for r in ranks])
+    cand = torch.stack([r.candidates(g) for r in ranks]).max(0).values
+    return [r.finish(cand) for r in ranks]
+
+
+def lockstep_verify(vs, slices_p, slices_q, tok, und, tree, shards, T):
+    ranks = [vs.ShardedVerify(p, q, tok, und, tree, s, T) for p, q, (s, _) in zip(slices_p, slices_q, shards)]
+    g = torch.stack([r.stats() for r in ranks])
+    gs = torch.stack([r.sums(g) for r in ranks])
+    tokmax = torch.stack([r.decide(gs) for r in ranks]).max(0).values
+    return [r.walk(tokmax.clone()) for r in ranks]
+
+
+@pytest.mark.parametrize("paper", [False, True])
+@pytest.mark.parametrize("nranks", [1, 2, 3, 8])
+@pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (9001, "bf16"), (40000, "bf16")])
+def test_sharded_matches_oracle(sh, V, dtype, nranks, paper):
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    lp, lq, un = make_case(V, dtype, V + nranks)
+    B, N, _ = lp.shape
+    T = np.array([1.0, 0.6, 1.3, 0.8], np.float32)
+    Tt = torch.from_numpy(T).cuda()
+    tp, tq, und = workloads.to_device(lp, dtype), workloads.to_device(lq, dtype), torch.from_numpy(un).cuda()
+    tree = sh.Tree.heap(N, leaves_sample=paper)
+    kind = workloads.paper_node_kind(N) if paper else None
+    shards = vs.even_shards(V, nranks)
+    # views into the full rows: slice starts are unaligned whenever an offset is odd
+    sp = [tp[:, :, s.id_offset:s.id_offset + w] for s, w in shards]
+    sq = [tq[:, :, s.id_offset:s.id_offset + w] for s, w in shards]
+
+    drafts = lockstep_draft(vs, sq, und, tree, shards, Tt)
+    for d in drafts[1:]:
+        for k in d:
+            assert torch.equal(d[k], drafts[0][k]), "ranks disagree on draft %s" % k
+    d0 = parity.to_numpy(drafts[0])
+    d0["prob"] = None
+    _, od = parity.check_draft("spechub", lq, T, un, d0, label="sharded-draft-%d" % nranks)
+
+    tok = torch.from_numpy(od["tokens"].copy()).cuda()
+    outs = lockstep_verify(vs, sp, sq, tok, und, tree, shards, Tt)
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        for k in o:
+            a, b = o[k], outs[0][k]
+            assert torch.equal(a.view(torch.int32) if a.dtype == torch.float32 else a,
+                               b.view(torch.int32) if b.dtype == torch.float32 else b), "ranks disagree on %s" % k
+    out = parity.to_numpy(outs[0])
+    assert (out["token"] >= -1).all(), "a drawn token was not delivered by its owner"
+    parity.check_verify("spechub", lp, lq, T, od["tokens"], un, kind, out, label="sharded-verify-%d" % nranks)
+    w = oracle.walk(out["accept_idx"], out["token"], tree.levels, node_kind=kind)
+    for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+        np.testing.assert_array_equal(out[k], w[k], err_msg="walk %s" % k)
+
+
+def test_one_rank_equals_the_unsharded_calls(sh):
+    """With a single rank the phases see the whole row: decisions and tokens equal the one-call path."""
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    lp, lq, un = make_case(5000, "fp32", 77)
+    tp, tq, und = workloads.to_device(lp, "fp32"), workloads.to_device(lq, "fp32"), torch.from_numpy(un).cuda()
+    tree = sh.Tree.heap(7)
+    shards = vs.even_shards(5000, 1)
+    d = lockstep_draft(vs, [tq], und, tree, shards, 1.0)[0]
+    ref = sh.spechub_draft_sample(tq, und, tree, 1.0)
+    for k in ("tokens", "hub", "status"):
+        assert torch.equal(d[k], ref[k]), k
+    o = lockstep_verify(vs, [tp], [tq], ref["tokens"], und, tree, shards, 1.0)[0]
+    full = sh.spechub_verify_tree(tp, tq, ref["tokens"], und, tree, 1.0)
+    for k in ("accept_idx", "token", "hub", "status", "n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+        assert torch.equal(o[k], full[k]), k
+    for k in ("beta", "rate"):
+        torch.testing.assert_close(o[k], full[k], rtol=1e-5, atol=1e-6)
+
+
+def test_shard_argument_errors(sh):
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    tq = torch.zeros((1, 3, 64), device="cuda")
+    un = torch.zeros((1, 3, 5), device="cuda")
+    tree = sh.Tree.heap(3)
+    for bad in (vs.Shard(2, 2, 0, 128), vs.Shard(0, 65, 0, 128), vs.Shard(0, 2, 100, 128), vs.Shard(0, 1, -1, 64)):
+        with pytest.raises(sh.SpecHubError):
+            vs.ShardedDraft(tq, un, tree, bad, 1.0).stats()
