@@ -132,7 +132,8 @@ __global__ void __launch_bounds__(512) shard_stats_kernel(ShardArgs a) {
         rec[0] = P.ml; rec[1] = P.sx;
         rec[2] = __int_as_float(P.ml > neg_inf() ? P.idx + a.id_offset : 0x7fffffff);
     }
-    const bool leaf = a.r.node_kind && a.r.node_kind[w.n] == SPECHUB_NODE_LEAF;
+    // verification reads no q on a leaf row; the draft step (no target given) drafts on every row
+    const bool leaf = a.r.target && a.r.node_kind && a.r.node_kind[w.n] == SPECHUB_NODE_LEAF;
     if (a.r.draft && !leaf) {
         const LT *rowq = static_cast<const LT *>(a.r.draft) + w.b * a.r.stride_seq + w.n * a.r.stride_node;
         const ArgMaxSum Q = pass_a<LT, AL>(g, rowq, w.k, sh.q);
