@@ -69,6 +69,7 @@ extern "C" {
 #define SPECHUB_ERR_WORKSPACE (-7)   /* workspace smaller than spechub_workspace_bytes()   */
 #define SPECHUB_ERR_LAUNCH (-8)      /* the CUDA runtime refused a launch                  */
 #define SPECHUB_ERR_METHOD (-9)      /* without_replacement is not 0 or 1                  */
+#define SPECHUB_ERR_TOO_LARGE (-10)  /* more rows than spechub_verify_tree_static can hold */
 
 /* logits element type */
 #define SPECHUB_F32 0
@@ -300,6 +301,40 @@ int spechub_shard_draft(const spechub_desc *desc, const spechub_shard *shard, co
 int spechub_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard,
                                const float *gathered_stats, const int32_t *cand_max,
                                int32_t *draft_tokens, int32_t *hub, uint32_t *status, void *stream);
+
+/*
+ * SpecHub verification and tree walk for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: this is a property of the library,
+ * not of the method.)  Inference servers that reserve the whole GPU for their
+ * own pools at start-up, code running inside another framework's memory plan,
+ * and real-time loops that may not enter the driver's allocator all fall in
+ * this class: for them every cudaMalloc is either forbidden or a stall.  This
+ * call runs the phase kernels of the vocabulary-sharded path as a single rank
+ * that holds the whole vocabulary -- stats, sums, decide, walk, back to back
+ * on `stream` -- and keeps the two per-row records those phases hand to one
+ * another (64 bytes per row) in a static array inside the library instead of
+ * buffers somebody would have to allocate.  It calls no cudaMalloc, cudaFree or
+ * other allocating routine.  Inputs and outputs are the caller's, with the
+ * meaning they have in spechub_verify_tree (desc->k must be 2; seq_out may be
+ * NULL); results equal spechub_verify_tree's up to fp32 summation order.
+ *
+ * Limits and rules:
+ *   - batch * nodes <= SPECHUB_STATIC_MAX_ROWS, else SPECHUB_ERR_TOO_LARGE and
+ *     nothing is launched.  The array takes SPECHUB_STATIC_MAX_ROWS * 64 bytes
+ *     (1 MiB) of every GPU that loads the library, until the process exits.
+ *   - The first call on each device looks the array's device address up (with
+ *     that device current) and keeps it; make that first call outside any
+ *     stream capture.  A failed look-up returns SPECHUB_ERR_LAUNCH.
+ *   - All calls on a device share the array.  Each call rewrites every record
+ *     it reads, so nothing has to be cleared and a call never sees another
+ *     call's leftovers; but two calls that overlap on the GPU (different
+ *     streams, no dependency between them) race on it.  Order them.
+ */
+#define SPECHUB_STATIC_MAX_ROWS 16384
+int spechub_verify_tree_static(const spechub_desc *desc, const void *target_logits,
+                               const void *draft_logits, const int32_t *draft_tokens,
+                               const float *uniforms, const spechub_node_out *node_out,
+                               const spechub_seq_out *seq_out, void *stream);
 
 /* Scratch bytes the two verify calls need for this descriptor (0 is possible). */
 size_t spechub_workspace_bytes(const spechub_desc *desc);

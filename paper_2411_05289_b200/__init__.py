@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     set_row_split,
     spechub_draft_sample,
     spechub_verify_tree,
+    spechub_verify_tree_static,
     status_string,
     workspace_bytes,
 )

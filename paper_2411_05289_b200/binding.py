@@ -102,6 +102,9 @@ def load_library(build_if_missing: bool = True):
     lib.mdsd_compare_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp,
                                              ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
                                              ctypes.c_size_t, vp]
+    lib.spechub_verify_tree_static.restype = i32
+    lib.spechub_verify_tree_static.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp,
+                                               ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp]
     lib.spechub_workspace_bytes.restype = ctypes.c_size_t
     lib.spechub_workspace_bytes.argtypes = [ctypes.POINTER(_Desc)]
     lib.spechub_status_string.restype = ctypes.c_char_p
@@ -395,6 +398,37 @@ def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
     _check(lib.mdsd_compare_verify_tree(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), tp,
                                         _ptr(uniforms), no, so, _ptr(ws), ws_bytes, _stream_ptr(stream)))
+    return out
+
+
+STATIC_MAX_ROWS = 16384
+
+
+def spechub_verify_tree_static(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
+                               temperature=1.0, stream=None, out=None):
+    """SpecHub verification and tree walk through the entry point that allocates nothing on the
+    device: for callers whose GPU memory is spoken for (a server's pre-reserved pools, another
+    framework's memory plan) or who may not enter the allocator at all.  The library keeps its
+    intermediate per-row records in a static array of its own, so at most ``STATIC_MAX_ROWS``
+    (batch x nodes) rows per call, and calls on one device must not overlap.  Pass ``out`` (from
+    ``alloc_verify_outputs``) to keep this wrapper from allocating the result tensors too."""
+    lib = load_library()
+    _need_k2(tree)
+    _same_layout(target_logits, draft_logits)
+    d, keep = _desc(target_logits, tree, temperature)
+    B, N, _ = target_logits.shape
+    dev = target_logits.device
+    _check_uniforms(uniforms, B, N, dev)
+    if (draft_tokens.dtype != torch.int32 or tuple(draft_tokens.shape) != (B, N, 2)
+            or not draft_tokens.is_contiguous() or draft_tokens.device != dev):
+        raise ValueError("draft_tokens must be a contiguous int32 [batch][nodes][2] tensor")
+    if out is None:
+        out = alloc_verify_outputs(B, N, tree.levels, dev)
+    no = _NodeOut(*[out[k].data_ptr() for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
+    so = _SeqOut(*[out[k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])
+    _check(lib.spechub_verify_tree_static(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits),
+                                          _ptr(draft_tokens), _ptr(uniforms), ctypes.byref(no),
+                                          ctypes.byref(so), _stream_ptr(stream)))
     return out
 
 

@@ -4,6 +4,8 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "spechub.h"
 #include "spechub_common.cuh"
 #include "spechub_stream.cuh"
@@ -505,6 +507,7 @@ const char *spechub_status_string(int code) {
         case SPECHUB_ERR_WORKSPACE: return "workspace smaller than spechub_workspace_bytes()";
         case SPECHUB_ERR_LAUNCH: return "kernel launch failed";
         case SPECHUB_ERR_METHOD: return "without_replacement must be 0 or 1";
+        case SPECHUB_ERR_TOO_LARGE: return "batch * nodes exceeds SPECHUB_STATIC_MAX_ROWS of spechub_verify_tree_static";
         default: return "unknown status";
     }
 }
@@ -512,3 +515,71 @@ const char *spechub_status_string(int code) {
 int spechub_abi_version(void) { return SPECHUB_ABI_VERSION; }
 
 }  // extern "C"
+
+// ---- verification without any allocation ---------------------------------------------------------
+// Scratch of spechub_verify_tree_static: per row the "stats" record and the "sums" record of the
+// phase kernels (8 floats each).  Lives in every GPU that loads the library until the process ends.
+static __device__ __align__(256) float g_static_scratch[(size_t)SPECHUB_STATIC_MAX_ROWS * 2 * spechub::kShardRecord];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float *g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, never an address a kernel may be given, so the address is looked up
+// once per device (with that device current) and kept.
+int static_scratch(float **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECHUB_ERR_LAUNCH;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SPECHUB_ERR_LAUNCH;
+        }
+        g_static_ptr[dev] = static_cast<float *>(p);
+    }
+    *out = g_static_ptr[dev];
+    return SPECHUB_OK;
+}
+
+}  // namespace
+
+extern "C" int spechub_verify_tree_static(const spechub_desc *desc, const void *target_logits,
+                                          const void *draft_logits, const int32_t *draft_tokens,
+                                          const float *uniforms, const spechub_node_out *no,
+                                          const spechub_seq_out *so, void *stream) {
+    const int rc = check_desc(desc);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->k != 2) return SPECHUB_ERR_SHAPE;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !no || !no->accept_idx || !no->token)
+        return SPECHUB_ERR_NULL;
+    const int64_t rows = desc->batch * (int64_t)desc->nodes;
+    if (rows > SPECHUB_STATIC_MAX_ROWS) return SPECHUB_ERR_TOO_LARGE;
+    float *scratch = nullptr;
+    const int src = static_scratch(&scratch);
+    if (src != SPECHUB_OK) return src;
+    float *stats = scratch, *sums = scratch + rows * kShardRecord;
+
+    // one rank that holds the whole vocabulary: the phase kernels, back to back on the stream
+    spechub_shard whole = {0, 1, 0, desc->vocab};
+    ShardArgs a = shard_args(desc, &whole);
+    a.r.target = target_logits; a.r.draft = draft_logits; a.r.draft_tokens_in = draft_tokens;
+    a.r.uniforms = uniforms;
+    a.out = stats;                     // every record is written in full: nothing has to start at zero
+    int prc = run_shard_phase(kPhaseStats, desc, a, stream);
+    if (prc != SPECHUB_OK) return prc;
+    a.gstats = stats; a.out = sums;
+    prc = run_shard_phase(kPhaseSums, desc, a, stream);
+    if (prc != SPECHUB_OK) return prc;
+    a.gsums = sums; a.out = nullptr;
+    a.r.hub = no->hub; a.r.accept_idx = no->accept_idx; a.r.token = no->token;
+    a.r.beta = no->beta; a.r.rate = no->rate; a.r.status = no->status;
+    prc = run_shard_phase(kPhaseDecide, desc, a, stream);
+    if (prc != SPECHUB_OK) return prc;
+    return launch_walk(desc, no, so, static_cast<cudaStream_t>(stream));
+}
