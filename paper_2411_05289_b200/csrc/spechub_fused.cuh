@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     merge_slices<1>(sh, 1, k, Q);
     const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
     const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
+    const float rho = __fdiv_rn(Zp, Zq);
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
     auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
     auto draw_from_p = [&]() { return lean_sample_row<1>(g, rowp, k, P, 0, -1, ures, 0, sh); };
@@ -125,6 +126,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     if (!ok_r[1]) o[2].status = SPECHUB_ST_TOKEN_RANGE;
     const bool degenerate = !(Q.sx > 0.f);
     const float c = degenerate ? 0.f : 1.f / Q.sx;
+    const float crho = c * rho;
     const float qa = invZq, rest = Q.sx * invZq;
     const int hubvec = hubtok >> 3, hubel = hubtok & 7;
     const int wx1 = ok_r[1] ? rx1[1] : -1;            // RRSw's first draft (left out of its renormaliser)
@@ -138,13 +140,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         float fp[8], fq[8];
         unpack_bf16x8(vp[vi], fp);
         unpack_bf16x8(vq[vi], fq);
-        float pp[8], qq[8];
+        float pp[8], qq[8];   // e_p, e_q (lean_terms: everything below is in units of 1 / Z_p)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
+        for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
 #pragma unroll
         for (int i = 0; i < 8; i += 2) {
-            a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
-            a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
+            a1a += fmaxf(__fmaf_rn(-rho, qq[i], pp[i]), 0.f);
+            a1b += fmaxf(__fmaf_rn(-rho, qq[i + 1], pp[i + 1]), 0.f);
         }
         {
             float qw[8];
@@ -166,19 +168,22 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
 #pragma unroll
         for (int i = 0; i < 8; i += 2) {
             float d, t;
-            transport_terms(pp[i], qq[i], c, d, t);
+            lean_terms(pp[i], qq[i], rho, crho, d, t);
             s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
-            transport_terms(pp[i + 1], qq[i + 1], c, d, t);
+            lean_terms(pp[i + 1], qq[i + 1], rho, crho, d, t);
             s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
         }
     }
     float accB[5] = {s1a + s1b, s2a + s2b, ra + rb, a1a + a1b, dna + dnb};
     lean_block_sums<5, 0>(accB, sh);   // per-warp R stays in sh.acc[2]
-    const float S1 = accB[0], S2 = degenerate ? qa : accB[1], R = accB[2], A1 = accB[3], den = accB[4];
+    const float Rraw = accB[2];
+    const float S1 = accB[0] * invZp, S2 = degenerate ? qa : accB[1] * invZp, R = Rraw * invZp;
+    const float A1 = accB[3] * invZp, den = accB[4] * invZq;
 
     // ---- pass C (forwards): second-stage residual masses of RRS and RRSw ----
     const bool q1_zero = !(den > 0.f);
     const float A1g[2] = {A1, A1 * (q1_zero ? 0.f : 1.f / den)};
+    const float A1grho[2] = {A1g[0] * rho, A1g[1] * rho};
     float w0a = 0.f, w0b = 0.f, w1a = 0.f, w1b = 0.f;
 #pragma unroll 2
     for (int vi = lo + lane; vi < hi; vi += 32) {
@@ -187,7 +192,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         unpack_bf16x8(vq[vi], fq);
         float sc[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) sc[i] = A1g[1];
+        for (int i = 0; i < 8; ++i) sc[i] = A1grho[1];
         if (vi == wvec) {
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -195,13 +200,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         }
 #pragma unroll
         for (int i = 0; i < 8; i += 2) {
-            const float p0 = prob_of(fp[i], k, cP, invZp), q0 = prob_of(fq[i], k, cQ, invZq);
-            const float p1 = prob_of(fp[i + 1], k, cP, invZp), q1 = prob_of(fq[i + 1], k, cQ, invZq);
+            const float p0 = lean_exp(fp[i], k, cP), q0 = lean_exp(fq[i], k, cQ);
+            const float p1 = lean_exp(fp[i + 1], k, cP), q1 = lean_exp(fq[i + 1], k, cQ);
             float d, t;
-            transport_terms(p0, q0, A1g[0], d, t); w0a += fmaxf(t, 0.f);
-            transport_terms(p1, q1, A1g[0], d, t); w0b += fmaxf(t, 0.f);
-            transport_terms(p0, q0, sc[i], d, t); w1a += fmaxf(t, 0.f);
-            transport_terms(p1, q1, sc[i + 1], d, t); w1b += fmaxf(t, 0.f);
+            lean_terms(p0, q0, rho, A1grho[0], d, t); w0a += fmaxf(t, 0.f);
+            lean_terms(p1, q1, rho, A1grho[0], d, t); w0b += fmaxf(t, 0.f);
+            lean_terms(p0, q0, rho, sc[i], d, t); w1a += fmaxf(t, 0.f);
+            lean_terms(p1, q1, rho, sc[i + 1], d, t); w1b += fmaxf(t, 0.f);
         }
     }
     float accC[2] = {w0a + w0b, w1a + w1b};
@@ -233,7 +238,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         if (!(acc1 || acc2)) {
             s.accept_idx = -1;
             int tok;
-            if (R > 0.f) {
+            if (Rraw > 0.f) {
                 if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[2][threadIdx.x];
                 __syncthreads();
                 auto wf = [&](int vi, float(&w)[8]) {
@@ -243,11 +248,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         float d, t;
-                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                        lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, crho, d, t);
                         w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
                     }
                 };
-                tok = block_sample3(g, wf, sh, ures * R);
+                tok = block_sample3(g, wf, sh, ures * Rraw);
             } else {
                 s.status |= SPECHUB_ST_ZERO_RESIDUAL;
                 tok = draw_from_p();
@@ -261,7 +266,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         if (!ok_r[m]) continue;
         NodeResult &s = o[1 + m];
         const bool wo = (m == 1);
-        const float W2 = accC[m];
+        const float W2raw = accC[m], W2 = W2raw * invZp;
         const int x1 = rx1[m], x2 = rx2[m];
         s.rate[0] = fmaxf(1.f - A1, 0.f);
         s.rate[1] = fmaxf(A1 - W2, 0.f);
@@ -279,10 +284,10 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         if (!(acc1 || acc2)) {
             s.accept_idx = -1;
             int tok;
-            if (A1 > 0.f && W2 > 0.f) {
+            if (A1 > 0.f && W2raw > 0.f) {
                 if (threadIdx.x < g.nwarps) sh.mass[threadIdx.x] = sh.acc[5 + m][threadIdx.x];
                 __syncthreads();
-                const float coef = A1g[m];
+                const float coef = A1grho[m];
                 auto wf = [&](int vi, float(&w)[8]) {
                     float fp[8], fq[8];
                     unpack_bf16x8(vp[vi], fp);
@@ -291,11 +296,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
                     for (int i = 0; i < 8; ++i) {
                         float d, t;
                         const float sc = (wo && vi * 8 + i == x1) ? 0.f : coef;
-                        transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc, d, t);
+                        lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, sc, d, t);
                         w[i] = fmaxf(t, 0.f);
                     }
                 };
-                tok = block_sample3(g, wf, sh, ures * W2);
+                tok = block_sample3(g, wf, sh, ures * W2raw);
             } else {
                 s.status |= SPECHUB_ST_ZERO_RESIDUAL;
                 tok = draw_from_p();

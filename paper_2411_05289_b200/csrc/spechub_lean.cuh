@@ -544,6 +544,16 @@ __device__ __forceinline__ void lean_row_sums(float (&x)[NACC], float (&part)[NA
     }
 }
 
+// Passes B and C work on the exponentials themselves, in units of 1 / Z_p: with rho = Z_p / Z_q,
+//   d = e_p - rho e_q = Z_p (p - q),   t = max(d, 0) - s rho e_q = Z_p (max(p - q, 0) - s q),
+// two FMAs per vocabulary pair instead of two multiplications by 1/Z, a subtraction and an FMA.
+// Identical target and draft rows give rho = 1 and e_p = e_q bit for bit, so d = 0 exactly.
+__device__ __forceinline__ float lean_exp(float logit, float k, float c) { return ex2(__fmaf_rn(logit, k, -c)); }
+__device__ __forceinline__ void lean_terms(float ep, float eq, float rho, float srho, float &d, float &t) {
+    d = __fmaf_rn(-rho, eq, ep);
+    t = __fmaf_rn(-srho, eq, fmaxf(d, 0.f));
+}
+
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
@@ -593,6 +603,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     merge_slices<CS>(sh, 1, k, Q);
     const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
     const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
+    const float rho = __fdiv_rn(Zp, Zq);
     const int x1 = a.draft_tokens_in[2 * r], x2 = a.draft_tokens_in[2 * r + 1];
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
     auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
@@ -619,6 +630,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
             const bool degenerate = !(Q.sx > 0.f);
             const float c = degenerate ? 0.f : 1.f / Q.sx;
+            const float crho = c * rho;
             const float qa = invZq, rest = Q.sx * invZq;
             const int hubvec = hubtok >> 3, hubel = hubtok & 7;
             const float px = prob_p(x), qx = prob_q(x);
@@ -650,16 +662,18 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 #pragma unroll
                 for (int i = 0; i < 8; i += 2) {
                     float d, t;
-                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                    lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, crho, d, t);
                     s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
-                    transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), c, d, t);
+                    lean_terms(lean_exp(fp[i + 1], k, cP), lean_exp(fq[i + 1], k, cQ), rho, crho, d, t);
                     s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
                 }
             }
             float acc[3] = {s1a + s1b, s2a + s2b, ra + rb};
             float part[3][CS];
             lean_row_sums<CS, 3, 0>(acc, part, sh);  // [2]
-            const float S1 = acc[0], S2 = degenerate ? qa : acc[1], R = acc[2];
+            // the sums are in units of 1 / Z_p; Rraw stays in them for the residual draw
+            const float Rraw = acc[2];
+            const float S1 = acc[0] * invZp, S2 = degenerate ? qa : acc[1] * invZp, R = Rraw * invZp;
             const float pa = prob_p(hubtok);
             const float hub_left = fmaxf(pa - S2, 0.f);
             o.rate[0] = fmaxf(rest - S1, 0.f) + fminf(pa, S2);
@@ -681,7 +695,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             if (!(acc1 || acc2)) {
                 o.accept_idx = -1;
                 float base = 0.f;
-                const int sel = (R > 0.f) ? pick_part(part[2], CS, ures * R, base) : -1;
+                const int sel = (Rraw > 0.f) ? pick_part(part[2], CS, ures * Rraw, base) : -1;
                 if (sel < 0) {
                     o.status |= SPECHUB_ST_ZERO_RESIDUAL;
                     draw_from_p();
@@ -697,11 +711,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 float d, t;
-                                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), c, d, t);
+                                lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, crho, d, t);
                                 w[i] = (vi * 8 + i == hubtok) ? 0.f : fmaxf(t, 0.f);
                             }
                         };
-                        const int tok = block_sample3(g, wf, sh, ures * R - base);
+                        const int tok = block_sample3(g, wf, sh, ures * Rraw - base);
                         if (threadIdx.x == 0) a.token[r] = tok;
                     }
                 }
@@ -725,13 +739,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 float fp[8], fq[8];
                 unpack_bf16x8(vp[vi], fp);
                 unpack_bf16x8(vq[vi], fq);
-                float pp[8], qq[8];
+                float pp[8], qq[8];   // e_p, e_q
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { pp[i] = prob_of(fp[i], k, cP, invZp); qq[i] = prob_of(fq[i], k, cQ, invZq); }
+                for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
 #pragma unroll
                 for (int i = 0; i < 8; i += 2) {
-                    a1a += fmaxf(__fsub_rn(pp[i], qq[i]), 0.f);
-                    a1b += fmaxf(__fsub_rn(pp[i + 1], qq[i + 1]), 0.f);
+                    a1a += fmaxf(__fmaf_rn(-rho, qq[i], pp[i]), 0.f);
+                    a1b += fmaxf(__fmaf_rn(-rho, qq[i + 1], pp[i + 1]), 0.f);
                 }
                 if (METHOD == kRRSw) {
                     if (vi == x1vec) {
@@ -746,10 +760,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             float acc[2] = {a1a + a1b, dna + dnb};
             float part2[2][CS];
             lean_row_sums<CS, 2, 0>(acc, part2, sh);  // [2]
-            const float A1 = acc[0], den = acc[1];
+            const float A1 = acc[0] * invZp, den = acc[1] * invZq;   // the sums are of exponentials
             const bool q1_zero = (METHOD == kRRSw) && !(den > 0.f);
             const float gq = (METHOD == kRRSw) ? (q1_zero ? 0.f : 1.f / den) : 1.f;
             const float A1g = A1 * gq;
+            const float A1grho = A1g * rho;
             // pass C: mass of the residual after two rejections
             float w2a = 0.f, w2b = 0.f;
 #pragma unroll 2
@@ -759,7 +774,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 unpack_bf16x8(vq[vi], fq);
                 float sc[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sc[i] = A1g;
+                for (int i = 0; i < 8; ++i) sc[i] = A1grho;
                 if (METHOD == kRRSw && vi == x1vec) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
@@ -768,16 +783,16 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 #pragma unroll
                 for (int i = 0; i < 8; i += 2) {
                     float d, t;
-                    transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), sc[i], d, t);
+                    lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, sc[i], d, t);
                     w2a += fmaxf(t, 0.f);
-                    transport_terms(prob_of(fp[i + 1], k, cP, invZp), prob_of(fq[i + 1], k, cQ, invZq), sc[i + 1], d, t);
+                    lean_terms(lean_exp(fp[i + 1], k, cP), lean_exp(fq[i + 1], k, cQ), rho, sc[i + 1], d, t);
                     w2b += fmaxf(t, 0.f);
                 }
             }
             float w2[1] = {w2a + w2b};
             float part1[1][CS];
             lean_row_sums<CS, 1, 2>(w2, part1, sh);  // [3]
-            const float W2 = w2[0];
+            const float W2raw = w2[0], W2 = W2raw * invZp;
             o.rate[0] = fmaxf(1.f - A1, 0.f);
             o.rate[1] = fmaxf(A1 - W2, 0.f);
             o.rate[2] = W2;
@@ -794,7 +809,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             if (!(acc1 || acc2)) {
                 o.accept_idx = -1;
                 float base = 0.f;
-                const int sel = (A1 > 0.f && W2 > 0.f) ? pick_part(part1[0], CS, ures * W2, base) : -1;
+                const int sel = (A1 > 0.f && W2raw > 0.f) ? pick_part(part1[0], CS, ures * W2raw, base) : -1;
                 if (sel < 0) {
                     o.status |= SPECHUB_ST_ZERO_RESIDUAL;
                     draw_from_p();
@@ -810,12 +825,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 float d, t;
-                                const float s = (METHOD == kRRSw && vi * 8 + i == x1) ? 0.f : A1g;
-                                transport_terms(prob_of(fp[i], k, cP, invZp), prob_of(fq[i], k, cQ, invZq), s, d, t);
+                                const float s = (METHOD == kRRSw && vi * 8 + i == x1) ? 0.f : A1grho;
+                                lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, s, d, t);
                                 w[i] = fmaxf(t, 0.f);
                             }
                         };
-                        const int tok = block_sample3(g, wf, sh, ures * W2 - base);
+                        const int tok = block_sample3(g, wf, sh, ures * W2raw - base);
                         if (threadIdx.x == 0) a.token[r] = tok;
                     }
                 }
