@@ -303,6 +303,37 @@ int spechub_shard_draft_finish(const spechub_desc *desc, const spechub_shard *sh
                                int32_t *draft_tokens, int32_t *hub, uint32_t *status, void *stream);
 
 /*
+ * RRS / RRSw (Algorithm 1, k = 2) on vocabulary-sharded logits: the phases above
+ * for the comparison methods.  As with SpecHub the paper has no counterpart.
+ *   verify: spechub_shard_stats -> all-gather -> rrs_shard_sums(gathered_sums =
+ *           NULL): A1 and RRSw's renormaliser over the slice, p and q at x1, x2
+ *           from their owners -> all-gather -> rrs_shard_sums(gathered_sums):
+ *           the second-stage residual mass W2 over the slice -> all-gather ->
+ *           rrs_shard_decide -> maximum of node_out->token -> spechub_walk_tree.
+ *   draft:  spechub_shard_stats(target = NULL) -> all-gather ->
+ *           rrs_shard_draft(cand_max = ex1_max = NULL): x1 ~ q and, for RRS, x2 ~ q
+ *           (each -2 where another rank draws); ex1 [B][N] = the exponential of
+ *           x1's logit on the row's scale from its owner, -1 elsewhere -> maximum
+ *           of cand and of ex1 over ranks -> RRSw only: rrs_shard_draft(cand_max,
+ *           ex1_max): x2 ~ q with q(x1) set to 0 -> maximum of cand ->
+ *           rrs_shard_draft_finish.
+ * out, gathered_*: as for SpecHub ([B][N][8] and [nranks][B][N][8] floats).
+ */
+int rrs_shard_sums(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                   const void *target_slice, const void *draft_slice, const int32_t *draft_tokens,
+                   const float *gathered_stats, const float *gathered_sums, float *out, void *stream);
+int rrs_shard_decide(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                     const void *target_slice, const void *draft_slice, const int32_t *draft_tokens,
+                     const float *uniforms, const float *gathered_stats, const float *gathered_sums,
+                     const float *gathered_w2, const spechub_node_out *node_out, void *stream);
+int rrs_shard_draft(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                    const void *draft_slice, const float *uniforms, const float *gathered_stats,
+                    const int32_t *cand_max, const float *ex1_max, int32_t *cand, float *ex1, void *stream);
+int rrs_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                           const float *gathered_stats, const int32_t *cand_max, int32_t *draft_tokens,
+                           uint32_t *status, void *stream);
+
+/*
  * SpecHub verification and tree walk for callers that cannot allocate device
  * memory.  (The paper has no counterpart: this is a property of the library,
  * not of the method.)  Inference servers that reserve the whole GPU for their

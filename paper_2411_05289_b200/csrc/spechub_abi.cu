@@ -13,6 +13,7 @@
 #include "spechub_kary.cuh"
 #include "spechub_fused.cuh"
 #include "spechub_shard.cuh"
+#include "spechub_shard_rrs.cuh"
 
 namespace {
 
@@ -335,14 +336,17 @@ ShardArgs shard_args(const spechub_desc *d, const spechub_shard *sh) {
     return a;
 }
 
-enum ShardPhase { kPhaseStats, kPhaseSums, kPhaseDecide, kPhaseDraft };
+enum ShardPhase { kPhaseStats, kPhaseSums, kPhaseDecide, kPhaseDraft, kPhaseRrsSums, kPhaseRrsDecide, kPhaseRrsDraft };
 
 template <typename LT, bool AL>
 void launch_shard_phase(int phase, const ShardArgs &a, unsigned rows, int th, cudaStream_t s) {
     if (phase == kPhaseStats) shard_stats_kernel<LT, AL><<<rows, th, 0, s>>>(a);
     else if (phase == kPhaseSums) shard_sums_kernel<LT, AL><<<rows, th, 0, s>>>(a);
     else if (phase == kPhaseDecide) shard_decide_kernel<LT, AL><<<rows, th, 0, s>>>(a);
-    else shard_draft_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else if (phase == kPhaseDraft) shard_draft_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else if (phase == kPhaseRrsSums) rrs_shard_sums_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else if (phase == kPhaseRrsDecide) rrs_shard_decide_kernel<LT, AL><<<rows, th, 0, s>>>(a);
+    else rrs_shard_draft_kernel<LT, AL><<<rows, th, 0, s>>>(a);
 }
 
 int run_shard_phase(int phase, const spechub_desc *d, const ShardArgs &a, void *stream) {
@@ -487,6 +491,74 @@ int spechub_shard_draft_finish(const spechub_desc *desc, const spechub_shard *sh
     a.gstats = gathered_stats; a.cand = cand_max;
     a.r.draft_tokens_out = draft_tokens; a.r.hub = hub; a.r.status = status;
     shard_draft_finish_kernel<<<(unsigned)((a.rows + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    return launch_status();
+}
+
+int rrs_shard_sums(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                   const void *target_slice, const void *draft_slice, const int32_t *draft_tokens,
+                   const float *gathered_stats, const float *gathered_sums, float *out, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!target_slice || !draft_slice || !draft_tokens || !gathered_stats || !out) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.without_replacement = without_replacement;
+    a.r.target = target_slice; a.r.draft = draft_slice; a.r.draft_tokens_in = draft_tokens;
+    a.gstats = gathered_stats; a.gsums = gathered_sums; a.out = out;
+    return run_shard_phase(kPhaseRrsSums, desc, a, stream);
+}
+
+int rrs_shard_decide(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                     const void *target_slice, const void *draft_slice, const int32_t *draft_tokens,
+                     const float *uniforms, const float *gathered_stats, const float *gathered_sums,
+                     const float *gathered_w2, const spechub_node_out *no, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!target_slice || !draft_slice || !draft_tokens || !uniforms || !gathered_stats || !gathered_sums ||
+        !gathered_w2 || !no || !no->accept_idx || !no->token)
+        return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.without_replacement = without_replacement;
+    a.r.target = target_slice; a.r.draft = draft_slice; a.r.draft_tokens_in = draft_tokens;
+    a.r.uniforms = uniforms; a.gstats = gathered_stats; a.gsums = gathered_sums; a.gw2 = gathered_w2;
+    a.r.hub = no->hub; a.r.accept_idx = no->accept_idx; a.r.token = no->token;
+    a.r.beta = no->beta; a.r.rate = no->rate; a.r.status = no->status;
+    return run_shard_phase(kPhaseRrsDecide, desc, a, stream);
+}
+
+int rrs_shard_draft(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                    const void *draft_slice, const float *uniforms, const float *gathered_stats,
+                    const int32_t *cand_max, const float *ex1_max, int32_t *cand, float *ex1, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!draft_slice || !uniforms || !gathered_stats || !cand) return SPECHUB_ERR_NULL;
+    if ((cand_max == nullptr) != (ex1_max == nullptr)) return SPECHUB_ERR_NULL;
+    if (cand_max && !without_replacement) return SPECHUB_ERR_METHOD;   // only RRSw has a second round
+    ShardArgs a = shard_args(desc, shard);
+    a.without_replacement = without_replacement;
+    a.r.draft = draft_slice; a.r.uniforms = uniforms; a.gstats = gathered_stats;
+    a.x1_known = cand_max; a.ex1_known = ex1_max; a.cand_out = cand; a.ex1_out = ex1;
+    return run_shard_phase(kPhaseRrsDraft, desc, a, stream);
+}
+
+int rrs_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard, int without_replacement,
+                           const float *gathered_stats, const int32_t *cand_max, int32_t *draft_tokens,
+                           uint32_t *status, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    const int rc = check_shard(desc, shard);
+    if (rc != SPECHUB_OK) return rc;
+    if (desc->batch == 0) return SPECHUB_OK;
+    if (!gathered_stats || !cand_max || !draft_tokens) return SPECHUB_ERR_NULL;
+    ShardArgs a = shard_args(desc, shard);
+    a.without_replacement = without_replacement;
+    a.gstats = gathered_stats; a.cand = cand_max;
+    a.r.draft_tokens_out = draft_tokens; a.r.status = status;
+    rrs_shard_draft_finish_kernel<<<(unsigned)((a.rows + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(a);
     return launch_status();
 }
 

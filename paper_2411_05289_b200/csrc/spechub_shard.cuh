@@ -26,6 +26,11 @@ struct ShardArgs {
     long long rows;
     const float *gstats;   // [nranks][rows][8]: (ml, sx, idx) of p then of q, per rank
     const float *gsums;    // [nranks][rows][8]
+    const float *gw2;      // [nranks][rows][8] (RRS / RRSw: second-stage residual masses)
+    int without_replacement;
+    const int32_t *x1_known;  // RRSw draft, second round: [rows][2] candidates after the maximum
+    const float *ex1_known;   // ... and the exponential of x1's logit, [rows]
+    float *ex1_out;           // first round: that exponential from x1's owner, -1 elsewhere
     const int32_t *cand;   // [rows][2] after the element-wise maximum over ranks
     float *out;            // [rows][8] phase output
     int32_t *cand_out;     // [rows][2]
@@ -140,6 +145,9 @@ __global__ void __launch_bounds__(512) shard_stats_kernel(ShardArgs a) {
         rec[4] = Q.ml; rec[5] = Q.sx;
         rec[6] = __int_as_float(Q.ml > neg_inf() ? Q.idx + a.id_offset : 0x7fffffff);
     }
+    // spare lanes: this slice's id range, so that every rank can tell which slice holds a given token
+    rec[3] = __int_as_float(a.id_offset);
+    rec[7] = __int_as_float(a.r.vocab);
     if (threadIdx.x < kShardRecord) a.out[w.r * kShardRecord + threadIdx.x] = rec[threadIdx.x];
 }
 

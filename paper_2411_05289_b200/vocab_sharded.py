@@ -64,6 +64,14 @@ def _lib():
         lib.spechub_shard_draft.argtypes = [D, S, vp, vp, vp, vp, vp]
         lib.spechub_shard_draft_finish.restype = i32
         lib.spechub_shard_draft_finish.argtypes = [D, S, vp, vp, vp, vp, vp, vp]
+        lib.rrs_shard_sums.restype = i32
+        lib.rrs_shard_sums.argtypes = [D, S, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.rrs_shard_decide.restype = i32
+        lib.rrs_shard_decide.argtypes = [D, S, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(_b._NodeOut), vp]
+        lib.rrs_shard_draft.restype = i32
+        lib.rrs_shard_draft.argtypes = [D, S, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.rrs_shard_draft_finish.restype = i32
+        lib.rrs_shard_draft_finish.argtypes = [D, S, i32, vp, vp, vp, vp, vp]
         _configured = True
     return lib
 
@@ -170,6 +178,78 @@ class ShardedVerify(_Phases):
         return self.out
 
 
+class ShardedRrsDraft(ShardedDraft):
+    """One rank's side of the RRS / RRSw draft step (RRSw takes a second round: `second`)."""
+
+    def __init__(self, draft_slice, uniforms, tree, shard, without_replacement, temperature=1.0, stream=None):
+        super().__init__(draft_slice, uniforms, tree, shard, temperature, stream)
+        self.wo = int(bool(without_replacement))
+
+    def candidates(self, gathered_stats):
+        """-> (cand [B][N][2] int32, ex1 [B][N] float32); take the maximum of both over ranks."""
+        _gathered_ok(gathered_stats, self.shard, self.B, self.N)
+        self.gstats = gathered_stats
+        cand = self._new((self.B, self.N, 2), torch.int32)
+        ex1 = self._new((self.B, self.N), torch.float32)
+        _b._check(self.lib.rrs_shard_draft(ctypes.byref(self.desc), ctypes.byref(self.cshard), self.wo,
+                                           _b._ptr(self.draft), _b._ptr(self.uniforms), _b._ptr(gathered_stats),
+                                           None, None, _b._ptr(cand), _b._ptr(ex1), self._sp()))
+        return cand, ex1
+
+    def second(self, cand_max, ex1_max):
+        """RRSw: x2 ~ q without x1 -> cand [B][N][2]; take the maximum over ranks again."""
+        cand = self._new((self.B, self.N, 2), torch.int32)
+        _b._check(self.lib.rrs_shard_draft(ctypes.byref(self.desc), ctypes.byref(self.cshard), self.wo,
+                                           _b._ptr(self.draft), _b._ptr(self.uniforms), _b._ptr(self.gstats),
+                                           _b._ptr(cand_max.contiguous()), _b._ptr(ex1_max.contiguous()),
+                                           _b._ptr(cand), None, self._sp()))
+        return cand
+
+    def finish(self, cand_max):
+        tokens = self._new((self.B, self.N, 2), torch.int32)
+        status = self._new((self.B, self.N), torch.int32)
+        _b._check(self.lib.rrs_shard_draft_finish(ctypes.byref(self.desc), ctypes.byref(self.cshard), self.wo,
+                                                  _b._ptr(self.gstats), _b._ptr(cand_max.contiguous()),
+                                                  _b._ptr(tokens), _b._ptr(status), self._sp()))
+        return dict(tokens=tokens, status=status)
+
+
+class ShardedRrsVerify(ShardedVerify):
+    """One rank's side of RRS / RRSw verification: stats, sums, w2, decide, walk."""
+
+    def __init__(self, target_slice, draft_slice, draft_tokens, uniforms, tree, shard, without_replacement,
+                 temperature=1.0, stream=None):
+        super().__init__(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, temperature, stream)
+        self.wo = int(bool(without_replacement))
+
+    def _sums(self, gathered_sums):
+        out = self._new((self.B, self.N, 8), torch.float32)
+        _b._check(self.lib.rrs_shard_sums(ctypes.byref(self.desc), ctypes.byref(self.cshard), self.wo,
+                                          _b._ptr(self.target), _b._ptr(self.draft), _b._ptr(self.tokens),
+                                          _b._ptr(self.gstats), _b._ptr(gathered_sums), _b._ptr(out), self._sp()))
+        return out
+
+    def sums(self, gathered_stats):
+        _gathered_ok(gathered_stats, self.shard, self.B, self.N)
+        self.gstats = gathered_stats
+        return self._sums(None)
+
+    def w2(self, gathered_sums):
+        _gathered_ok(gathered_sums, self.shard, self.B, self.N)
+        self.gsums = gathered_sums
+        return self._sums(gathered_sums)
+
+    def decide(self, gathered_w2):
+        _gathered_ok(gathered_w2, self.shard, self.B, self.N)
+        self.out = _b.alloc_verify_outputs(self.B, self.N, self.tree.levels, self.dev)
+        no = _b._NodeOut(*[self.out[k].data_ptr() for k in ("accept_idx", "token", "hub", "beta", "rate", "status")])
+        _b._check(self.lib.rrs_shard_decide(ctypes.byref(self.desc), ctypes.byref(self.cshard), self.wo,
+                                            _b._ptr(self.target), _b._ptr(self.draft), _b._ptr(self.tokens),
+                                            _b._ptr(self.uniforms), _b._ptr(self.gstats), _b._ptr(self.gsums),
+                                            _b._ptr(gathered_w2), ctypes.byref(no), self._sp()))
+        return self.out["token"]
+
+
 # ---- the collectives -----------------------------------------------------------------------------
 
 def all_gather_ranks(t, group=None):
@@ -212,3 +292,22 @@ def spechub_verify_tree_sharded(target_slice, draft_slice, draft_tokens, uniform
     v = ShardedVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, temperature, stream)
     gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
     return v.walk(all_max(v.decide(gsums), group))
+
+
+def rrs_draft_sample_sharded(draft_slice, uniforms, tree, shard: Shard, without_replacement, temperature=1.0,
+                             group=None, stream=None):
+    d = ShardedRrsDraft(draft_slice, uniforms, tree, shard, without_replacement, temperature, stream)
+    cand, ex1 = d.candidates(all_gather_ranks(d.stats(), group))
+    cand, ex1 = all_max(cand, group), all_max(ex1, group)
+    if without_replacement:
+        cand = all_max(d.second(cand, ex1), group)
+    return d.finish(cand)
+
+
+def rrs_verify_tree_sharded(target_slice, draft_slice, draft_tokens, uniforms, tree, shard: Shard,
+                            without_replacement, temperature=1.0, group=None, stream=None):
+    v = ShardedRrsVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, without_replacement,
+                         temperature, stream)
+    gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
+    gw2 = all_gather_ranks(v.w2(gsums), group)
+    return v.walk(all_max(v.decide(gw2), group))

@@ -22,6 +22,7 @@ def test_header_declares_the_expected_entry_points():
         "mdsd_compare_draft_sample", "mdsd_compare_verify_tree", "spechub_walk_tree",
         "spechub_shard_stats", "spechub_shard_sums", "spechub_shard_decide", "spechub_shard_draft",
         "spechub_shard_draft_finish", "spechub_verify_tree_static",
+        "rrs_shard_sums", "rrs_shard_decide", "rrs_shard_draft", "rrs_shard_draft_finish",
         "spechub_workspace_bytes", "spechub_status_string", "spechub_abi_version"])
 
 

@@ -97,6 +97,68 @@ def test_sharded_matches_oracle(sh, V, dtype, nranks, paper):
         np.testing.assert_array_equal(out[k], w[k], err_msg="walk %s" % k)
 
 
+def lockstep_rrs_draft(vs, slices_q, und, tree, shards, T, wo):
+    ranks = [vs.ShardedRrsDraft(q, und, tree, s, wo, T) for q, (s, _) in zip(slices_q, shards)]
+    g = torch.stack([r.stats() for r in ranks])
+    res = [r.candidates(g) for r in ranks]
+    cand = torch.stack([c for c, _ in res]).max(0).values
+    ex1 = torch.stack([e for _, e in res]).max(0).values
+    if wo:
+        cand = torch.stack([r.second(cand, ex1) for r in ranks]).max(0).values
+    return [r.finish(cand) for r in ranks]
+
+
+def lockstep_rrs_verify(vs, slices_p, slices_q, tok, und, tree, shards, T, wo):
+    ranks = [vs.ShardedRrsVerify(p, q, tok, und, tree, s, wo, T) for p, q, (s, _) in zip(slices_p, slices_q, shards)]
+    g = torch.stack([r.stats() for r in ranks])
+    gs = torch.stack([r.sums(g) for r in ranks])
+    gw = torch.stack([r.w2(gs) for r in ranks])
+    tokmax = torch.stack([r.decide(gw) for r in ranks]).max(0).values
+    return [r.walk(tokmax.clone()) for r in ranks]
+
+
+@pytest.mark.parametrize("wo", [False, True])
+@pytest.mark.parametrize("paper", [False, True])
+@pytest.mark.parametrize("nranks", [1, 3, 8])
+@pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (9001, "bf16"), (40000, "bf16")])
+def test_sharded_rrs_matches_oracle(sh, V, dtype, nranks, paper, wo):
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    method = "rrsw" if wo else "rrs"
+    lp, lq, un = make_case(V, dtype, V + nranks + 100)
+    B, N, _ = lp.shape
+    T = np.array([1.0, 0.6, 1.3, 0.8], np.float32)
+    Tt = torch.from_numpy(T).cuda()
+    tp, tq, und = workloads.to_device(lp, dtype), workloads.to_device(lq, dtype), torch.from_numpy(un).cuda()
+    tree = sh.Tree.heap(N, leaves_sample=paper)
+    kind = workloads.paper_node_kind(N) if paper else None
+    shards = vs.even_shards(V, nranks)
+    sp = [tp[:, :, s.id_offset:s.id_offset + w] for s, w in shards]
+    sq = [tq[:, :, s.id_offset:s.id_offset + w] for s, w in shards]
+
+    drafts = lockstep_rrs_draft(vs, sq, und, tree, shards, Tt, wo)
+    for d in drafts[1:]:
+        for k in d:
+            assert torch.equal(d[k], drafts[0][k]), "ranks disagree on draft %s" % k
+    d0 = parity.to_numpy(drafts[0])
+    _, od = parity.check_draft(method, lq, T, un, d0, label="sharded-%s-draft-%d" % (method, nranks))
+
+    tok = torch.from_numpy(od["tokens"].copy()).cuda()
+    outs = lockstep_rrs_verify(vs, sp, sq, tok, und, tree, shards, Tt, wo)
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        for k in o:
+            a, b = o[k], outs[0][k]
+            assert torch.equal(a.view(torch.int32) if a.dtype == torch.float32 else a,
+                               b.view(torch.int32) if b.dtype == torch.float32 else b), "ranks disagree on %s" % k
+    out = parity.to_numpy(outs[0])
+    assert (out["token"] >= -1).all(), "a drawn token was not delivered by its owner"
+    parity.check_verify(method, lp, lq, T, od["tokens"], un, kind, out, label="sharded-%s-verify-%d" % (method, nranks))
+    w = oracle.walk(out["accept_idx"], out["token"], tree.levels, node_kind=kind)
+    for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+        np.testing.assert_array_equal(out[k], w[k], err_msg="walk %s" % k)
+
+
 def test_one_rank_equals_the_unsharded_calls(sh):
     """With a single rank the phases see the whole row: decisions and tokens equal the one-call path."""
     from paper_2411_05289_b200 import vocab_sharded as vs
