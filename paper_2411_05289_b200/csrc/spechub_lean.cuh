@@ -246,9 +246,9 @@ __device__ void lean_reduce2(const LeanAcc &tp, const LeanAcc &tq, const uint4 *
 
 // CTA-wide inverse-CDF draw over this CTA's part of a row.  sh.mass[w] = total weight of warp w's
 // range (the coarse CDF); weights(vi, w[8]) the weights of vector vi; t = target prefix within
-// this part.  Every thread knows the selected warp range; round 1 cuts it into one contiguous
+// this part.  Every thread knows the selected warp range; pass 1 cuts it into one contiguous
 // block of vectors per thread of the CTA and sums the blocks in parallel, warp 0 scans the block
-// sums; round 2 spreads the chosen block's vectors over the lanes of warp 0.  Two load round trips
+// sums; pass 2 spreads the chosen block's vectors over the lanes of warp 0.  Two load round trips
 // in all.  Returns to every thread the lowest id whose inclusive prefix exceeds t; when rounding
 // leaves none inside the selected range, the last id with positive weight there; -1 when this
 // part has no mass.  Called by all threads of the CTA.
@@ -270,7 +270,7 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) 
     if (wsel < 0) { wsel = lastw; base = lastbase; }
     const int lo = g.seg_lo(wsel), hi = g.seg_hi(wsel);
     const int Bv = (hi - lo + nth - 1) / nth;  // vectors per thread block
-    {   // round 1
+    {   // pass 1
         const int b0 = lo + threadIdx.x * Bv, b1 = min(hi, b0 + Bv);
         float tot = 0.f;
 #pragma unroll 4
@@ -323,7 +323,7 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) 
         blk = sh.blk;
         tt2 = sh.tt2;
         int found = -1;
-        if (blk >= 0) {   // round 2: the block's vectors over the lanes
+        if (blk >= 0) {   // pass 2: the block's vectors over the lanes
             const int c0 = lo + blk * Bv, c1 = min(hi, c0 + Bv);
             float prefix = 0.f;
             int lastpos = -1;

@@ -3,8 +3,8 @@
 // SpecHub's, because the second-stage residual mass W2 depends on the row-wide A1; the draft step
 // without replacement needs a second round, because q without x1 is known only once x1 is.
 //
-//   sums (round 1)  A1 = sum max(p - q, 0) over the slice; RRSw: sum of q outside x1; p, q at x1, x2
-//   sums (round 2)  W2 = sum max(max(p - q, 0) - A1 q1, 0) over the slice
+//   sums (1st call) A1 = sum max(p - q, 0) over the slice; RRSw: sum of q outside x1; p, q at x1, x2
+//   sums (2nd call) W2 = sum max(max(p - q, 0) - A1 q1, 0) over the slice
 //   decide          Algorithm 1's two tests; residual token by the rank that holds the target
 //   draft           x1 ~ q; x2 ~ q (RRS, same round) or ~ q without x1 (RRSw, second round)
 #pragma once
@@ -198,8 +198,8 @@ __global__ void __launch_bounds__(512) rrs_shard_decide_kernel(ShardArgs a) {
     if (threadIdx.x == 0) write_node(a.r, w.r, o);
 }
 
-// Draft rounds.  Round 1 (x1_known == NULL): x1 ~ q, RRS also x2 ~ q; x1's owner publishes the
-// exponential of its logit.  Round 2 (RRSw): x2 ~ q with q(x1) set to 0.
+// Draft calls.  First call (x1_known == NULL): x1 ~ q, RRS also x2 ~ q; x1's owner publishes the
+// exponential of its logit.  Second call (RRSw): x2 ~ q with q(x1) set to 0.
 template <typename LT, bool AL>
 __global__ void __launch_bounds__(512) rrs_shard_draft_kernel(ShardArgs a) {
     constexpr int VW = VecOf<LT>::W;
