@@ -249,6 +249,44 @@ def test_argument_errors(sh):
     assert out["tokens"].shape == (0, 3, 2)
 
 
+@pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (9001, "bf16"), (12344, "bf16"), (40000, "bf16")])
+def test_strided_views_equal_contiguous_rows(sh, V, dtype):
+    """Rows taken out of a larger buffer (gaps between nodes and between sequences, a base that
+    is not the allocation's start) give bit for bit what the same rows give when contiguous."""
+    rng = np.random.default_rng(V + 41)
+    B, N = 4, 7
+    lp, lq = random_logits(rng, B, N, V, dtype)
+    un = random_uniforms(rng, B, N)
+    und = torch.from_numpy(un).cuda()
+    tp, tq = workloads.to_device(lp, dtype), workloads.to_device(lq, dtype)
+    Vp = (V + 15) // 16 * 16 + 16
+
+    def embed(t):
+        big = torch.full((B + 1, N + 3, Vp), float("nan"), dtype=t.dtype, device="cuda")
+        view = big[1:, 2:N + 2, 8:8 + V]
+        view.copy_(t)
+        return view
+
+    sp, sq = embed(tp), embed(tq)
+    assert not sp.is_contiguous() and sp.stride(2) == 1
+    tree = sh.Tree.heap(N)
+    for m in METHODS:
+        d_ref = gpu_draft(sh, m, tq, und, tree, 1.0)
+        d_str = gpu_draft(sh, m, sq, und, tree, 1.0)
+        assert torch.equal(d_ref["tokens"], d_str["tokens"]) and torch.equal(d_ref["status"], d_str["status"])
+        ref = gpu_verify(sh, m, tp, tq, d_ref["tokens"], und, tree, 1.0)
+        got = gpu_verify(sh, m, sp, sq, d_ref["tokens"], und, tree, 1.0)
+        for k in ref:
+            a, b = ref[k], got[k]
+            if a.dtype == torch.float32:
+                a, b = a.view(torch.int32), b.view(torch.int32)
+            assert torch.equal(a, b), "%s %s" % (m, k)
+    all3 = sh.mdsd_compare_verify_tree(sp, sq, {m: gpu_draft(sh, m, tq, und, tree, 1.0)["tokens"] for m in METHODS},
+                                       und, tree, 1.0)
+    ref0 = gpu_verify(sh, "spechub", tp, tq, gpu_draft(sh, "spechub", tq, und, tree, 1.0)["tokens"], und, tree, 1.0)
+    assert torch.equal(all3["spechub"]["token"], ref0["token"])
+
+
 def test_custom_child_table_and_determinism(sh):
     rng = np.random.default_rng(21)
     B, N, V = 16, 5, 3000
