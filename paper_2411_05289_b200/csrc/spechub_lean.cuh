@@ -649,11 +649,16 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
             // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
             float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
-#pragma unroll 2
+            // software pipeline: the next vector pair is in registers before this one is consumed
+            uint4 np = make_uint4(0, 0, 0, 0), nq = np;
+            if (last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
+#pragma unroll 1
             for (int vi = last_vi; vi >= lo; vi -= 32) {
+                const uint4 cp = np, cq = nq;
+                if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
                 float fp[8], fq[8];
-                unpack_bf16x8(vp[vi], fp);
-                unpack_bf16x8(vq[vi], fq);
+                unpack_bf16x8(cp, fp);
+                unpack_bf16x8(cq, fq);
                 if (vi == hubvec) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
