@@ -76,9 +76,6 @@ constexpr int kLeanThreads = 256;  // 4 CTAs per SM measured best (256/512/1024:
 // read at any time; at CS = 4 on V = 128256 that fits L2 (DRAM reads drop from 2.0x to 1.0x the
 // algorithmic bytes) but the per-CTA fixed work grows 4x, and the two cancel (1.6 vs 1.8 ms).
 int lean_split(const spechub_desc *d) {
-#ifdef SPECHUB_TUNE
-    if (getenv("SPECHUB_CS")) return atoi(getenv("SPECHUB_CS"));
-#endif
     if (d->flags & SPECHUB_FLAG_SPLIT_1) return 1;
     if (d->flags & SPECHUB_FLAG_SPLIT_2) return 2;
     if (d->flags & SPECHUB_FLAG_SPLIT_4) return 4;

@@ -1,8 +1,8 @@
 // General streaming kernels: one CTA per (sequence, node) row, any vocabulary
-// size, fp32 or bf16 logits.  Pass A reads the row(s) from HBM; the later passes
-// re-read them, which hit L2 while the row pair is still resident there.  The
-// register-resident kernels in spechub_resident.cuh replace these where a row
-// fits on chip; these remain the path for every other shape.
+// size, fp32 or bf16 logits, aligned or not.  Pass A reads the row(s) from HBM;
+// the later passes re-read them, which hit L2 while the row pair is still
+// there.  Large bf16 vocabularies with aligned rows take the kernels of
+// spechub_lean.cuh instead; these remain the path for every other shape.
 #pragma once
 
 #include "spechub.h"
