@@ -739,11 +739,23 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
             const int x1vec = x1 >> 3, x1el = x1 & 7;
             float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
-#pragma unroll 2
+            // RRSw: the next vector pair is loaded before the current one is consumed (measured:
+            // 2.21 -> 2.03 ms on V = 128256; for RRS the plain loop unrolled twice is the faster one)
+            constexpr bool PIPE = (METHOD == kRRSw);
+            uint4 np = make_uint4(0, 0, 0, 0), nq = np;
+            if (PIPE && last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
+#pragma unroll(PIPE ? 1 : 2)
             for (int vi = last_vi; vi >= lo; vi -= 32) {
+                uint4 cp, cq;
+                if (PIPE) {
+                    cp = np; cq = nq;
+                    if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
+                } else {
+                    cp = vp[vi]; cq = vq[vi];
+                }
                 float fp[8], fq[8];
-                unpack_bf16x8(vp[vi], fp);
-                unpack_bf16x8(vq[vi], fq);
+                unpack_bf16x8(cp, fp);
+                unpack_bf16x8(cq, fq);
                 float pp[8], qq[8];   // e_p, e_q
 #pragma unroll
                 for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
@@ -772,11 +784,19 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             const float A1grho = A1g * rho;
             // pass C: mass of the residual after two rejections
             float w2a = 0.f, w2b = 0.f;
-#pragma unroll 2
+            if (PIPE && lo + lane < hi) { np = vp[lo + lane]; nq = vq[lo + lane]; }
+#pragma unroll(PIPE ? 1 : 2)
             for (int vi = lo + lane; vi < hi; vi += 32) {
+                uint4 cp, cq;
+                if (PIPE) {
+                    cp = np; cq = nq;
+                    if (vi + 32 < hi) { np = vp[vi + 32]; nq = vq[vi + 32]; }
+                } else {
+                    cp = vp[vi]; cq = vq[vi];
+                }
                 float fp[8], fq[8];
-                unpack_bf16x8(vp[vi], fp);
-                unpack_bf16x8(vq[vi], fq);
+                unpack_bf16x8(cp, fp);
+                unpack_bf16x8(cq, fq);
                 float sc[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) sc[i] = A1grho;
