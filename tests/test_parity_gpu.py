@@ -419,3 +419,38 @@ def test_config5_sampled(sh):
     extra = [(r, k) for k, rows in per_kind.items() for r in rows]
     s = sampled_parity(sh, cfg, 48, extra_rows=[e[0] for e in extra])
     print("c5 %r" % s)
+
+
+# ------------------------------------------------------------------------------------------------
+# extremes of the shape: very long rows, very many rows
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,dtype", [(1 << 20, "bf16"), ((1 << 20) + 3, "bf16"), (600_001, "fp32")])
+def test_very_long_rows(sh, V, dtype):
+    """A million-token vocabulary: index arithmetic and the two-level samplers at their far end."""
+    rng = np.random.default_rng(V % 1000)
+    lp, lq = random_logits(rng, 1, 3, V, dtype, sd=3.0)
+    lq[0, 1, V - 1] = lq[0, 1].max() + 4.0        # hub is the very last id
+    lp, lq = workloads.round_to_storage(lp, dtype), workloads.round_to_storage(lq, dtype)
+    un = random_uniforms(rng, 1, 3)
+    un[0, 2, 0] = np.float32(1.0 - 2.0 ** -24)    # the largest uniform: the draw lands at the end of the CDF
+    run_case(sh, lp, lq, dtype, 1.0, un, paper_layout=False, label="long-rows")
+
+
+def test_very_many_rows(sh):
+    """More rows than a 16-bit grid dimension holds; a sample of them against the oracle."""
+    rng = np.random.default_rng(9)
+    B, N, V = 70_001, 1, 24
+    lp, lq = random_logits(rng, B, N, V, "fp32")
+    un = random_uniforms(rng, B, N)
+    tp, tq, und = workloads.to_device(lp, "fp32"), workloads.to_device(lq, "fp32"), torch.from_numpy(un).cuda()
+    tree = sh.Tree.heap(1)
+    pick = np.unique(np.concatenate([[0, 65535, 65536, B - 1], rng.integers(0, B, 200)]))
+    for m in METHODS:
+        d = parity.to_numpy(gpu_draft(sh, m, tq, und, tree, 1.0))
+        dsub = {k: (v[pick] if v is not None else None) for k, v in d.items()}
+        _, od = parity.check_draft(m, lq[pick], 1.0, un[pick], dsub, label="many-rows")
+        out = parity.to_numpy(gpu_verify(sh, m, tp, tq, torch.from_numpy(d["tokens"]).cuda(), und, tree, 1.0))
+        osub = {k: v[pick] for k, v in out.items()}
+        parity.check_verify(m, lp[pick], lq[pick], 1.0, d["tokens"][pick], un[pick], None, osub, label="many-rows")
+        assert (out["n_emitted"] == (out["accept_idx"][:, 0] >= 0) + 1).all()
