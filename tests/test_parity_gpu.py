@@ -453,4 +453,6 @@ def test_very_many_rows(sh):
         out = parity.to_numpy(gpu_verify(sh, m, tp, tq, torch.from_numpy(d["tokens"]).cuda(), und, tree, 1.0))
         osub = {k: v[pick] for k, v in out.items()}
         parity.check_verify(m, lp[pick], lq[pick], 1.0, d["tokens"][pick], un[pick], None, osub, label="many-rows")
-        assert (out["n_emitted"] == (out["accept_idx"][:, 0] >= 0) + 1).all()
+        w = oracle.walk(out["accept_idx"], out["token"], 1)
+        for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+            np.testing.assert_array_equal(out[k], w[k], err_msg="many-rows walk %s" % k)
