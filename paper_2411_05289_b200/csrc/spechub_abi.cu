@@ -107,7 +107,7 @@ int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cuda
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
     if (cs == 2) return launch_group(lean_draft_kernel<kLeanThreads, 2>, 2, rows, s, a, method);
-    return launch_group(lean_draft_kernel<kLeanThreads, 1>, 1, rows, s, a, method);
+    return launch_group(lean_draft_ck_kernel<kLeanThreads>, 1, rows, s, a, method);
 }
 
 bool lean_ok(const spechub_desc *d, bool aligned) {

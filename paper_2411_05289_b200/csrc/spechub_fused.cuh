@@ -311,8 +311,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     finish();
 }
 
-// Draft step of the three methods from one read of q.  x1 ~ q is the same draw for all three
-// (they share u_d1).
+// Draft step of the three methods from one read of q (the checkpointed pass A and sampler of
+// lean_draft_ck_kernel).  x1 ~ q is the same draw for all three: they share u_d1.
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(FusedArgs A, int32_t *hub_out,
                                                                             float *draft_prob) {
@@ -328,9 +328,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
     const float k = kLog2e / temperature_of(a, b);
     const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
     const bool t0 = threadIdx.x == 0;
+    const int CK = lean_ck_interval(g);
 
     LeanAcc tq, unused;
-    lean_pass_a<false>(vq, vq, lo, hi, lane, k, tq, unused);
+    unused.m2 = 0xff80ff80u; unused.s = 0.f; unused.c = 0.f;
+    lean_pass_a_ck(vq, lo, hi, lane, k, CK, tq, sh.cks[warp], sh.ckc[warp]);
     {
         ArgMaxSum q, unusedq;
         lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
@@ -352,7 +354,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
         return;
     }
     const int hubtok = Q.idx;
-    const int x1 = lean_sample_row<1>(g, rowq, k, Q, 0, -1, u1, 0, sh);
+    const int x1 = lean_ck_sample(g, rowq, k, Q.C, CK, -1, u1, sh);
     uint32_t st[3] = {0, 0, 0};
     int x2[3];
     // SpecHub (Section 4)
@@ -365,21 +367,16 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
         x2[0] = (hubtok == 0) ? 1 : 0;
         st[0] |= SPECHUB_ST_DEGENERATE_Q;
     } else {
-        x2[0] = lean_sample_row<1>(g, rowq, k, Q, 0, hubtok, u2, 0, sh);
+        x2[0] = lean_ck_sample(g, rowq, k, Q.C, CK, hubtok, u2, sh);
         prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2[0]), k, -Q.C)) / Q.sx;
     }
     // RRS: an independent second draw
-    x2[1] = lean_sample_row<1>(g, rowq, k, Q, 0, -1, u2, 0, sh);
+    x2[1] = lean_ck_sample(g, rowq, k, Q.C, CK, -1, u2, sh);
     // RRSw: q with q(x1) set to 0
-    {
-        float m0 = slice_mass<1>(sh, 0, Q, 0, x1, k);
-        if (sh.x_idx[0] != x1) m0 = fmaxf(m0 - ex2(__fmaf_rn(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)), 0.f);
-        if (m0 > 0.f) {
-            x2[2] = lean_sample_slice(g, rowq, k, Q, x1, u2 * m0, 0, sh);
-        } else {
-            st[2] |= SPECHUB_ST_DEGENERATE_Q;
-            x2[2] = (x1 == 0) ? 1 : 0;
-        }
+    x2[2] = lean_ck_sample(g, rowq, k, Q.C, CK, x1, u2, sh);
+    if (x2[2] < 0) {
+        x2[2] = (x1 == 0) ? 1 : 0;
+        st[2] |= SPECHUB_ST_DEGENERATE_Q;
     }
     if (t0) {
         for (int m = 0; m < 3; ++m) {

@@ -36,6 +36,7 @@ namespace spechub {
 namespace cg = cooperative_groups;
 
 constexpr int kLeanMaxWarps = 32;
+constexpr int kLeanCk = 16;       // checkpoints per warp in the draft step's pass A
 constexpr float kHuge = 1.0e30f;  // ~2^100: partial sums beyond this move the reference
 
 struct LeanShared {
@@ -45,6 +46,10 @@ struct LeanShared {
     float acc[8][kLeanMaxWarps];
     float mass[kLeanMaxWarps];
     float part[1024];  // sampler: per-thread block sums of the selected warp range
+    // draft step: checkpoint sums of pass A (per warp, every CK lane-iterations), their exponent
+    // references, and the masses of those sub-blocks on the row's scale
+    float cks[kLeanMaxWarps][kLeanCk], ckc[kLeanMaxWarps][kLeanCk];
+    float ckm[kLeanMaxWarps * kLeanCk];
     float tt2;
     int blk;
     int tok;
@@ -252,23 +257,11 @@ __device__ void lean_reduce2(const LeanAcc &tp, const LeanAcc &tq, const uint4 *
 // in all.  Returns to every thread the lowest id whose inclusive prefix exceeds t; when rounding
 // leaves none inside the selected range, the last id with positive weight there; -1 when this
 // part has no mass.  Called by all threads of the CTA.
+// The two passes of the CTA-wide draw over the vectors [lo, hi): tt = target prefix within the
+// range.  Called by all threads of the CTA; returns the id to every thread (-1: no mass in range).
 template <class WF>
-__device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) {
+__device__ int range_sample3(int lo, int hi, WF weights, LeanShared &sh, float tt) {
     const int lane = threadIdx.x & 31, nth = blockDim.x;
-    int wsel = -1, lastw = -1;
-    float base = 0.f, lastbase = 0.f, run = 0.f;
-    for (int w = 0; w < g.nwarps; ++w) {
-        const float m = sh.mass[w];
-        if (m > 0.f) {
-            lastw = w;
-            lastbase = run;
-            if (wsel < 0 && run + m > t) { wsel = w; base = run; }
-        }
-        run += m;
-    }
-    if (lastw < 0) return -1;
-    if (wsel < 0) { wsel = lastw; base = lastbase; }
-    const int lo = g.seg_lo(wsel), hi = g.seg_hi(wsel);
     const int Bv = (hi - lo + nth - 1) / nth;  // vectors per thread block
     {   // pass 1
         const int b0 = lo + threadIdx.x * Bv, b1 = min(hi, b0 + Bv);
@@ -283,7 +276,6 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) 
     }
     __syncthreads();
     if (threadIdx.x < 32) {
-        const float tt = t - base;
         const int per = nth >> 5;  // block sums per lane
         float ls = 0.f;
         for (int i = 0; i < per; ++i) ls += sh.part[lane * per + i];
@@ -383,6 +375,24 @@ __device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) 
     const int tok = sh.tok;
     __syncthreads();
     return tok;
+}
+
+template <class WF>
+__device__ int block_sample3(const Geo &g, WF weights, LeanShared &sh, float t) {
+    int wsel = -1, lastw = -1;
+    float base = 0.f, lastbase = 0.f, run = 0.f;
+    for (int w = 0; w < g.nwarps; ++w) {
+        const float m = sh.mass[w];
+        if (m > 0.f) {
+            lastw = w;
+            lastbase = run;
+            if (wsel < 0 && run + m > t) { wsel = w; base = run; }
+        }
+        run += m;
+    }
+    if (lastw < 0) return -1;
+    if (wsel < 0) { wsel = lastw; base = lastbase; }
+    return range_sample3(g.seg_lo(wsel), g.seg_hi(wsel), weights, sh, t - base);
 }
 
 // Pick the CTA of a row whose part holds the target t of an inverse-CDF draw over per-CTA masses
@@ -989,6 +999,218 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
         }
     }
     if (CS > 1) RowGroup<CS>::sync();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Draft step, one CTA per row, with a finer coarse CDF.  Pass A records, every CK lane-iterations,
+// the warp's sum since its previous checkpoint: sub-blocks of 32 * CK consecutive vectors, at most
+// kLeanCk per warp.  A draw then picks a sub-block from those sums and rescans only that (a few KB
+// instead of a warp's whole range), which is what the two-pass sampler costs most.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int lean_ck_interval(const Geo &g) {
+    const int iters = (g.seg + 31) >> 5;
+    return max(4, (iters + kLeanCk - 1) / kLeanCk);
+}
+
+__device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, int lane, float k, int CK,
+                                               LeanAcc &Q, float *cks, float *ckc) {
+    LeanAcc st;
+    st.m2 = 0xff80ff80u; st.s = 0.f; st.c = 0.f;
+    {   // one exponent reference for the whole warp: the maximum of its first vectors
+        float m0 = neg_inf();
+        if (lo + lane < hi) {
+            const uint4 a = rq[lo + lane];
+            m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m0 = fmaxf(m0, __shfl_xor_sync(kFull, m0, o));
+        if (m0 > neg_inf()) st.c = shift_of(m0, k);
+    }
+    float tot = 0.f, ctot = st.c;   // this thread's sum over all checkpoints, on the scale ctot
+    const int iters = (hi - lo + 31) >> 5;
+    int j = 0;
+    for (int it0 = 0; it0 < iters; it0 += CK) {
+        const int it1 = min(iters, it0 + CK);
+#pragma unroll 2
+        for (int it = it0; it < it1; ++it) {
+            const int vi = lo + lane + 32 * it;
+            if (vi < hi) lean_push(st, rq[vi], k);
+        }
+        // checkpoint: the warp's sum since the last one.  A lane that had to move its reference
+        // (sums beyond 2^100, rare) is brought to the warp's largest reference first.
+        const float c0 = __shfl_sync(kFull, st.c, 0);
+        float contrib = st.s, cref = c0;
+        if (__any_sync(kFull, st.c != c0)) {
+            float cm = st.c;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, o));
+            contrib = st.s > 0.f ? st.s * ex2(st.c - cm) : 0.f;
+            cref = cm;
+        }
+        const float cs = warp_sum(contrib);
+        if (lane == 0) { cks[j] = cs; ckc[j] = cref; }
+        ++j;
+        if (st.c != ctot) { tot = tot > 0.f ? tot * ex2(ctot - st.c) : 0.f; ctot = st.c; }
+        tot += st.s;
+        st.s = 0.f;
+    }
+    if (lane == 0)
+        for (; j < kLeanCk; ++j) { cks[j] = 0.f; ckc[j] = 0.f; }
+    Q.m2 = st.m2; Q.c = st.c; Q.s = tot;
+}
+
+// Inverse-CDF draw from softmax(row) without token `excl` (excl < 0: nothing left out) over the
+// checkpoint sub-blocks.  C = the row's exponent shift.  Returns to every thread the token, -1 if
+// nothing has mass.  Called by all threads of the CTA, after the checkpoints are visible.
+__device__ int lean_ck_sample(const Geo &g, const __nv_bfloat16 *row, float k, float C, int CK, int excl,
+                              float u, LeanShared &sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nslot = g.nwarps * kLeanCk;
+    auto wf = [&](int vi, float(&w)[8]) {
+        float v[8];
+        load_vec<__nv_bfloat16, true>(row, vi, g.V, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
+    };
+    for (int s = threadIdx.x; s < nslot; s += blockDim.x) {
+        const float cs = sh.cks[s / kLeanCk][s % kLeanCk];
+        sh.ckm[s] = cs > 0.f ? cs * ex2(sh.ckc[s / kLeanCk][s % kLeanCk] - C) : 0.f;
+    }
+    __syncthreads();
+    if (excl >= 0) {
+        // the sub-block that holds the excluded token is summed again without it: subtracting the
+        // token's own term would cancel when that token carries most of the sub-block's mass
+        const int ev = excl >> 3;
+        const int w = g.warp_of_vec(ev), j = (ev - g.seg_lo(w)) / (32 * CK);
+        const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
+        float s = 0.f;
+        for (int vi = b0 + threadIdx.x; vi < b1; vi += blockDim.x) {
+            float wt[8];
+            wf(vi, wt);
+            s += ((wt[0] + wt[1]) + (wt[2] + wt[3])) + ((wt[4] + wt[5]) + (wt[6] + wt[7]));
+        }
+        s = warp_sum(s);
+        if (lane == 0) sh.mass[warp] = s;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float t = 0.f;
+            for (int x = 0; x < g.nwarps; ++x) t += sh.mass[x];
+            sh.ckm[w * kLeanCk + j] = t;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x < 32) {   // warp 0: prefix sums over the sub-blocks, in id order
+        const int per = (nslot + 31) >> 5;
+        float ls = 0.f;
+        for (int i = 0; i < per; ++i) {
+            const int s = lane * per + i;
+            if (s < nslot) ls += sh.ckm[s];
+        }
+        float incl = ls;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const float total = __shfl_sync(kFull, incl, 31);
+        const float t = u * total;
+        const unsigned pos = __ballot_sync(kFull, ls > 0.f);
+        const unsigned hit = __ballot_sync(kFull, ls > 0.f && incl > t);
+        if (!pos || !(total > 0.f)) {
+            if (lane == 0) sh.blk = -1;
+        } else {
+            const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
+            if (lane == L) {
+                float acc = incl - ls, lastacc = 0.f;
+                int sel = -1, last = -1;
+                for (int i = 0; i < per; ++i) {
+                    const int s = lane * per + i;
+                    const float m = s < nslot ? sh.ckm[s] : 0.f;
+                    if (m > 0.f) {
+                        last = s;
+                        lastacc = acc;
+                        if (sel < 0 && acc + m > t) { sel = s; sh.tt2 = t - acc; }
+                    }
+                    acc += m;
+                }
+                if (sel < 0) { sel = last; sh.tt2 = t - lastacc; }
+                sh.blk = sel;
+            }
+        }
+    }
+    __syncthreads();
+    const int slot = sh.blk;
+    const float tt = sh.tt2;
+    __syncthreads();   // range_sample3 reuses blk / tt2
+    if (slot < 0) return -1;
+    const int w = slot / kLeanCk, j = slot % kLeanCk;
+    const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
+    return range_sample3(b0, b1, wf, sh, tt);
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(RowArgs a, int method) {
+    __shared__ LeanShared sh;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vq = reinterpret_cast<const uint4 *>(rowq);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const float k = kLog2e / temperature_of(a, b);
+    const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
+    const int CK = lean_ck_interval(g);
+
+    LeanAcc tq, unused;
+    unused.m2 = 0xff80ff80u; unused.s = 0.f; unused.c = 0.f;
+    lean_pass_a_ck(vq, lo, hi, lane, k, CK, tq, sh.cks[warp], sh.ckc[warp]);
+    {
+        ArgMaxSum q, unusedq;
+        lean_reduce2<false>(tq, unused, vq, vq, lo, hi, k, sh, q, unusedq);
+        if (threadIdx.x == 0) { sh.x_ml[0] = q.ml; sh.x_sx[0] = q.sx; sh.x_idx[0] = q.idx; }
+    }
+    __syncthreads();
+    RowStat Q;
+    merge_slices<1>(sh, 0, k, Q);
+    const float Zq = Q.sx + 1.f;
+    uint32_t st = 0;
+    int x1 = -1, x2 = -1, hubtok = -1;
+    float prob0 = 0.f, prob1 = 0.f;
+    if (!(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf())) {
+        st = SPECHUB_ST_NONFINITE;
+    } else {
+        hubtok = Q.idx;
+        x1 = lean_ck_sample(g, rowq, k, Q.C, CK, -1, u1, sh);
+        if (method == kSpecHub) {
+            prob0 = 1.f / Zq;
+            if (x1 != hubtok) {
+                x2 = hubtok;
+                prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)) / Zq;
+            } else if (!(Q.sx > 0.f)) {
+                x2 = (hubtok == 0) ? 1 : 0;
+                st |= SPECHUB_ST_DEGENERATE_Q;
+            } else {
+                x2 = lean_ck_sample(g, rowq, k, Q.C, CK, hubtok, u2, sh);
+                prob1 = prob0 * ex2(fmaf(load_one<__nv_bfloat16>(rowq, x2), k, -Q.C)) / Q.sx;
+            }
+        } else if (method == kRRS) {
+            x2 = lean_ck_sample(g, rowq, k, Q.C, CK, -1, u2, sh);
+        } else {
+            x2 = lean_ck_sample(g, rowq, k, Q.C, CK, x1, u2, sh);
+            if (x2 < 0) {   // nothing left once x1 is removed
+                x2 = (x1 == 0) ? 1 : 0;
+                st |= SPECHUB_ST_DEGENERATE_Q;
+            }
+        }
+    }
+    if (threadIdx.x == 0) {
+        a.draft_tokens_out[2 * r] = x1;
+        a.draft_tokens_out[2 * r + 1] = x2;
+        if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;
+        if (a.draft_prob) { a.draft_prob[2 * r] = prob0; a.draft_prob[2 * r + 1] = prob1; }
+        if (a.status) a.status[r] = st;
+    }
 }
 
 }  // namespace spechub
