@@ -1009,7 +1009,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ int lean_ck_interval(const Geo &g) {
     const int iters = (g.seg + 31) >> 5;
-    return max(4, (iters + kLeanCk - 1) / kLeanCk);
+    return 4 * max(1, (iters + 4 * kLeanCk - 1) / (4 * kLeanCk));   // a multiple of the unroll of pass A
 }
 
 __device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, int lane, float k, int CK,
@@ -1026,34 +1026,45 @@ __device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, 
         for (int o = 16; o > 0; o >>= 1) m0 = fmaxf(m0, __shfl_xor_sync(kFull, m0, o));
         if (m0 > neg_inf()) st.c = shift_of(m0, k);
     }
+    float cref = st.c;              // the reference every lane is expected to hold
     float tot = 0.f, ctot = st.c;   // this thread's sum over all checkpoints, on the scale ctot
-    const int iters = (hi - lo + 31) >> 5;
     int j = 0;
-    for (int it0 = 0; it0 < iters; it0 += CK) {
-        const int it1 = min(iters, it0 + CK);
-#pragma unroll 2
-        for (int it = it0; it < it1; ++it) {
-            const int vi = lo + lane + 32 * it;
-            if (vi < hi) lean_push(st, rq[vi], k);
-        }
-        // checkpoint: the warp's sum since the last one.  A lane that had to move its reference
-        // (sums beyond 2^100, rare) is brought to the warp's largest reference first.
-        const float c0 = __shfl_sync(kFull, st.c, 0);
-        float contrib = st.s, cref = c0;
-        if (__any_sync(kFull, st.c != c0)) {
+    // checkpoint: the warp's sum since the last one.  A lane that had to move its reference (sums
+    // beyond 2^100, rare) is brought to the warp's largest reference first.
+    auto checkpoint = [&]() {
+        float contrib = st.s, cnow = cref;
+        if (__any_sync(kFull, st.c != cref)) {
             float cm = st.c;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, o));
             contrib = st.s > 0.f ? st.s * ex2(st.c - cm) : 0.f;
-            cref = cm;
+            cnow = cm;
         }
         const float cs = warp_sum(contrib);
-        if (lane == 0) { cks[j] = cs; ckc[j] = cref; }
+        if (lane == 0) { cks[j] = cs; ckc[j] = cnow; }
         ++j;
         if (st.c != ctot) { tot = tot > 0.f ? tot * ex2(ctot - st.c) : 0.f; ctot = st.c; }
         tot += st.s;
         st.s = 0.f;
+    };
+    const int iters = (hi - lo + 31) >> 5;   // lane-iterations of this warp
+    const int nfull = (hi - lo) >> 5;        // those in which every lane has a vector
+    const uint4 *p = rq + lo + lane;
+    int it = 0, since = 0;
+    for (; it + 4 <= nfull; it += 4) {
+        const uint4 a0 = p[32 * it], a1 = p[32 * (it + 1)], a2 = p[32 * (it + 2)], a3 = p[32 * (it + 3)];
+        lean_push(st, a0, k);
+        lean_push(st, a1, k);
+        lean_push(st, a2, k);
+        lean_push(st, a3, k);
+        since += 4;
+        if (since >= CK) { checkpoint(); since = 0; }
     }
+    for (; it < iters; ++it) {
+        if (lo + lane + 32 * it < hi) lean_push(st, p[32 * it], k);
+        if (++since >= CK) { checkpoint(); since = 0; }
+    }
+    if (since > 0) checkpoint();
     if (lane == 0)
         for (; j < kLeanCk; ++j) { cks[j] = 0.f; ckc[j] = 0.f; }
     Q.m2 = st.m2; Q.c = st.c; Q.s = tot;
