@@ -36,7 +36,7 @@ namespace spechub {
 namespace cg = cooperative_groups;
 
 constexpr int kLeanMaxWarps = 32;
-constexpr int kLeanCk = 16;       // checkpoints per warp in the draft step's pass A
+constexpr int kLeanCk = 8;        // checkpoints per warp in the draft step's pass A
 constexpr float kHuge = 1.0e30f;  // ~2^100: partial sums beyond this move the reference
 
 struct LeanShared {
@@ -1051,8 +1051,15 @@ __device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, 
     const int nfull = (hi - lo) >> 5;        // those in which every lane has a vector
     const uint4 *p = rq + lo + lane;
     int it = 0, since = 0;
+    // four vectors per lane in flight; the next four are requested before the current ones are
+    // consumed, so that the checkpoint's shuffle chain overlaps the loads
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0, n3 = n0;
+    if (4 <= nfull) { n0 = p[0]; n1 = p[32]; n2 = p[64]; n3 = p[96]; }
     for (; it + 4 <= nfull; it += 4) {
-        const uint4 a0 = p[32 * it], a1 = p[32 * (it + 1)], a2 = p[32 * (it + 2)], a3 = p[32 * (it + 3)];
+        const uint4 a0 = n0, a1 = n1, a2 = n2, a3 = n3;
+        if (it + 8 <= nfull) {
+            n0 = p[32 * (it + 4)]; n1 = p[32 * (it + 5)]; n2 = p[32 * (it + 6)]; n3 = p[32 * (it + 7)];
+        }
         lean_push(st, a0, k);
         lean_push(st, a1, k);
         lean_push(st, a2, k);
