@@ -70,6 +70,7 @@ RowArgs base_args(const spechub_desc *d) {
 
 // The lean kernels take bf16 rows whose starts are 16-byte aligned and whose length is a
 // multiple of 8 and large enough to keep 512 threads busy.
+constexpr int kLeanDraftThreads = 128;
 constexpr int kLeanThreads = 256;  // 4 CTAs per SM measured best (256/512/1024: 1.54/1.65/1.87 ms)
 
 // CTAs per row.  With 4 CTAs per SM and 148 SMs, 592/CS rows are between their first and second
@@ -107,7 +108,11 @@ int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cuda
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
     if (cs == 2) return launch_group(lean_draft_kernel<kLeanThreads, 2>, 2, rows, s, a, method);
-    return launch_group(lean_draft_ck_kernel<kLeanThreads>, 1, rows, s, a, method);
+    // one CTA per row: 128 threads, 8 CTAs per SM measured best for the single-pass draft step
+    // (64 / 128 / 256 / 512 threads: 0.41 / 0.36 / 0.38 / 0.52 ms on V = 128256; 0.078 / 0.081 / 0.102 /
+    // 0.165 ms on V = 32000)
+    lean_draft_ck_kernel<kLeanDraftThreads><<<rows, kLeanDraftThreads, 0, s>>>(a, method);
+    return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
 }
 
 bool lean_ok(const spechub_desc *d, bool aligned) {
@@ -270,7 +275,8 @@ int compare_draft(const spechub_desc *d, const void *draft_logits, const float *
         f.dstatus[m] = status ? status[m] : nullptr;
     }
     const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
-    fused_draft_kernel<kLeanThreads><<<rows, kLeanThreads, 0, static_cast<cudaStream_t>(stream)>>>(f, hub, draft_prob);
+    // same CTA shape as lean_draft_ck_kernel: the results are to be the same bit for bit
+    fused_draft_kernel<kLeanDraftThreads><<<rows, kLeanDraftThreads, 0, static_cast<cudaStream_t>(stream)>>>(f, hub, draft_prob);
     return launch_status();
 }
 
