@@ -14,7 +14,8 @@
  *   - All data pointers are DEVICE pointers owned by the caller, valid until
  *     the work enqueued on `stream` has finished.  The descriptor itself is
  *     read on the host during the call.  The library allocates nothing and
- *     keeps no state between calls.
+ *     keeps no state between calls (spechub_verify_tree_static alone holds a
+ *     static scratch array; see there).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls enqueue work and return without synchronising.
  *   - Return value: SPECHUB_OK (0) when the work was enqueued; a negative
@@ -81,7 +82,7 @@ extern "C" {
 #define SPECHUB_ST_DEGENERATE_Q 4u    /* draft mass outside the excluded token is 0 (one-hot q)    */
 #define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
 #define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
-#define SPECHUB_ST_INTERNAL 32u       /* a bounded wait for an on-chip copy expired: row output is -1 */
+#define SPECHUB_ST_INTERNAL 32u       /* reserved: no kernel of this version waits on anything that can time out */
 
 /* descriptor flags: how many CTAs of a thread-block cluster share one row in the large-vocabulary
  * bf16 kernels (a tuning hint; results do not depend on it beyond fp32 summation order).  At most
