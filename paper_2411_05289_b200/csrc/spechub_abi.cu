@@ -100,9 +100,24 @@ int launch_lean_verify_cs(int method, const RowArgs &a, unsigned rows, cudaStrea
     if (method == kRRS) return launch_group(lean_verify_kernel<kRRS, kLeanThreads, CS>, CS, rows, s, a);
     return launch_group(lean_verify_kernel<kRRSw, kLeanThreads, CS>, CS, rows, s, a);
 }
+// The leaf rows of an unsplit call (same CTA shape as the draft step).
+int launch_lean_leaf(const RowArgs &a, const NodeOutPtrs *outs, int n_out, unsigned rows, cudaStream_t s) {
+    LeafArgs la = {};
+    la.r = a;
+    la.n_out = n_out;
+    for (int m = 0; m < n_out; ++m) la.out[m] = outs[m];
+    lean_leaf_kernel<kLeanDraftThreads><<<rows, kLeanDraftThreads, 0, s>>>(la);
+    return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+}
+
 int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_lean_verify_cs<4>(method, a, rows, s);
     if (cs == 2) return launch_lean_verify_cs<2>(method, a, rows, s);
+    if (a.node_kind) {
+        const NodeOutPtrs o = {a.accept_idx, a.token, a.hub, a.beta, a.rate, a.status};
+        const int lrc = launch_lean_leaf(a, &o, 1, rows, s);
+        if (lrc != SPECHUB_OK) return lrc;
+    }
     return launch_lean_verify_cs<1>(method, a, rows, s);
 }
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
@@ -313,6 +328,10 @@ int compare_verify(const spechub_desc *d, const void *target_logits, const void 
     }
     const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (d->node_kind) {
+        const int llrc = launch_lean_leaf(f.r, f.out, 3, rows, s);
+        if (llrc != SPECHUB_OK) return llrc;
+    }
     fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
     int lrc = launch_status();
     for (int m = 0; m < 3 && lrc == SPECHUB_OK && so; ++m) lrc = launch_walk(d, &no[m], &so[m], s);

@@ -15,11 +15,6 @@
 
 namespace spechub {
 
-struct NodeOutPtrs {
-    int32_t *accept_idx, *token, *hub;
-    float *beta, *rate;
-    uint32_t *status;
-};
 struct FusedArgs {
     RowArgs r;                 // target, draft, uniforms, temperature, node_kind, shape
     const int32_t *tok[3];     // draft tokens of SpecHub, RRS, RRSw (verify)
@@ -69,13 +64,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         for (int m = 0; m < 3; ++m) write_node3(A.out[m], r, o[m], elsewhere[m]);
     };
 
+    if (leaf) return;   // leaf rows belong to lean_leaf_kernel
     LeanAcc tp, tq;
-    if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
-    else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
+    lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
     {
         ArgMaxSum Ps, Qs;
-        if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
-        else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
         if (t0) {
             sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
             sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
@@ -94,12 +88,6 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
 
     if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
         for (int m = 0; m < 3; ++m) o[m].status = SPECHUB_ST_NONFINITE;
-        finish();
-        return;
-    }
-    if (leaf) {
-        const int tok = draw_from_p();   // the three methods share u_res, so they share the bonus token
-        for (int m = 0; m < 3; ++m) { o[m].token = tok; o[m].rate[2] = 1.f; }
         finish();
         return;
     }

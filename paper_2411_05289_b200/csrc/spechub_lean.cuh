@@ -554,6 +554,225 @@ __device__ __forceinline__ void lean_row_sums(float (&x)[NACC], float (&part)[NA
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Draft step, one CTA per row, with a finer coarse CDF.  Pass A records, every CK lane-iterations,
+// the warp's sum since its previous checkpoint: sub-blocks of 32 * CK consecutive vectors, at most
+// kLeanCk per warp.  A draw then picks a sub-block from those sums and rescans only that (a few KB
+// instead of a warp's whole range), which is what the two-pass sampler costs most.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int lean_ck_interval(const Geo &g) {
+    const int iters = (g.seg + 31) >> 5;
+    return 4 * max(1, (iters + 4 * kLeanCk - 1) / (4 * kLeanCk));   // a multiple of the unroll of pass A
+}
+
+__device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, int lane, float k, int CK,
+                                               LeanAcc &Q, float *cks, float *ckc) {
+    LeanAcc st;
+    st.m2 = 0xff80ff80u; st.s = 0.f; st.c = 0.f;
+    {   // one exponent reference for the whole warp: the maximum of its first vectors
+        float m0 = neg_inf();
+        if (lo + lane < hi) {
+            const uint4 a = rq[lo + lane];
+            m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m0 = fmaxf(m0, __shfl_xor_sync(kFull, m0, o));
+        if (m0 > neg_inf()) st.c = shift_of(m0, k);
+    }
+    float cref = st.c;              // the reference every lane is expected to hold
+    float tot = 0.f, ctot = st.c;   // this thread's sum over all checkpoints, on the scale ctot
+    int j = 0;
+    // checkpoint: the warp's sum since the last one.  A lane that had to move its reference (sums
+    // beyond 2^100, rare) is brought to the warp's largest reference first.
+    auto checkpoint = [&]() {
+        float contrib = st.s, cnow = cref;
+        if (__any_sync(kFull, st.c != cref)) {
+            float cm = st.c;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, o));
+            contrib = st.s > 0.f ? st.s * ex2(st.c - cm) : 0.f;
+            cnow = cm;
+        }
+        const float cs = warp_sum(contrib);
+        if (lane == 0) { cks[j] = cs; ckc[j] = cnow; }
+        ++j;
+        if (st.c != ctot) { tot = tot > 0.f ? tot * ex2(ctot - st.c) : 0.f; ctot = st.c; }
+        tot += st.s;
+        st.s = 0.f;
+    };
+    const int iters = (hi - lo + 31) >> 5;   // lane-iterations of this warp
+    const int nfull = (hi - lo) >> 5;        // those in which every lane has a vector
+    const uint4 *p = rq + lo + lane;
+    int it = 0, since = 0;
+    // four vectors per lane in flight; the next four are requested before the current ones are
+    // consumed, so that the checkpoint's shuffle chain overlaps the loads
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0, n3 = n0;
+    if (4 <= nfull) { n0 = p[0]; n1 = p[32]; n2 = p[64]; n3 = p[96]; }
+    for (; it + 4 <= nfull; it += 4) {
+        const uint4 a0 = n0, a1 = n1, a2 = n2, a3 = n3;
+        if (it + 8 <= nfull) {
+            n0 = p[32 * (it + 4)]; n1 = p[32 * (it + 5)]; n2 = p[32 * (it + 6)]; n3 = p[32 * (it + 7)];
+        }
+        lean_push(st, a0, k);
+        lean_push(st, a1, k);
+        lean_push(st, a2, k);
+        lean_push(st, a3, k);
+        since += 4;
+        if (since >= CK) { checkpoint(); since = 0; }
+    }
+    for (; it < iters; ++it) {
+        if (lo + lane + 32 * it < hi) lean_push(st, p[32 * it], k);
+        if (++since >= CK) { checkpoint(); since = 0; }
+    }
+    if (since > 0) checkpoint();
+    if (lane == 0)
+        for (; j < kLeanCk; ++j) { cks[j] = 0.f; ckc[j] = 0.f; }
+    Q.m2 = st.m2; Q.c = st.c; Q.s = tot;
+}
+
+// Inverse-CDF draw from softmax(row) without token `excl` (excl < 0: nothing left out) over the
+// checkpoint sub-blocks.  C = the row's exponent shift.  Returns to every thread the token, -1 if
+// nothing has mass.  Called by all threads of the CTA, after the checkpoints are visible.
+__device__ int lean_ck_sample(const Geo &g, const __nv_bfloat16 *row, float k, float C, int CK, int excl,
+                              float u, LeanShared &sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nslot = g.nwarps * kLeanCk;
+    auto wf = [&](int vi, float(&w)[8]) {
+        float v[8];
+        load_vec<__nv_bfloat16, true>(row, vi, g.V, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
+    };
+    for (int s = threadIdx.x; s < nslot; s += blockDim.x) {
+        const float cs = sh.cks[s / kLeanCk][s % kLeanCk];
+        sh.ckm[s] = cs > 0.f ? cs * ex2(sh.ckc[s / kLeanCk][s % kLeanCk] - C) : 0.f;
+    }
+    __syncthreads();
+    if (excl >= 0) {
+        // the sub-block that holds the excluded token is summed again without it: subtracting the
+        // token's own term would cancel when that token carries most of the sub-block's mass
+        const int ev = excl >> 3;
+        const int w = g.warp_of_vec(ev), j = (ev - g.seg_lo(w)) / (32 * CK);
+        const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
+        float s = 0.f;
+        for (int vi = b0 + threadIdx.x; vi < b1; vi += blockDim.x) {
+            float wt[8];
+            wf(vi, wt);
+            s += ((wt[0] + wt[1]) + (wt[2] + wt[3])) + ((wt[4] + wt[5]) + (wt[6] + wt[7]));
+        }
+        s = warp_sum(s);
+        if (lane == 0) sh.mass[warp] = s;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float t = 0.f;
+            for (int x = 0; x < g.nwarps; ++x) t += sh.mass[x];
+            sh.ckm[w * kLeanCk + j] = t;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x < 32) {   // warp 0: prefix sums over the sub-blocks, in id order
+        const int per = (nslot + 31) >> 5;
+        float ls = 0.f;
+        for (int i = 0; i < per; ++i) {
+            const int s = lane * per + i;
+            if (s < nslot) ls += sh.ckm[s];
+        }
+        float incl = ls;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const float total = __shfl_sync(kFull, incl, 31);
+        const float t = u * total;
+        const unsigned pos = __ballot_sync(kFull, ls > 0.f);
+        const unsigned hit = __ballot_sync(kFull, ls > 0.f && incl > t);
+        if (!pos || !(total > 0.f)) {
+            if (lane == 0) sh.blk = -1;
+        } else {
+            const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
+            if (lane == L) {
+                float acc = incl - ls, lastacc = 0.f;
+                int sel = -1, last = -1;
+                for (int i = 0; i < per; ++i) {
+                    const int s = lane * per + i;
+                    const float m = s < nslot ? sh.ckm[s] : 0.f;
+                    if (m > 0.f) {
+                        last = s;
+                        lastacc = acc;
+                        if (sel < 0 && acc + m > t) { sel = s; sh.tt2 = t - acc; }
+                    }
+                    acc += m;
+                }
+                if (sel < 0) { sel = last; sh.tt2 = t - lastacc; }
+                sh.blk = sel;
+            }
+        }
+    }
+    __syncthreads();
+    const int slot = sh.blk;
+    const float tt = sh.tt2;
+    __syncthreads();   // range_sample3 reuses blk / tt2
+    if (slot < 0) return -1;
+    const int w = slot / kLeanCk, j = slot % kLeanCk;
+    const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
+    return range_sample3(b0, b1, wf, sh, tt);
+}
+
+// Leaf rows (Figure 2: after the last accepted draft the bonus token is a draw from p) of a call
+// whose rows are not split over clusters get a kernel of their own, shaped like the draft step:
+// pass A over p with checkpoints, then the sub-block sampler.  CTAs of verifying rows leave at
+// once; the verification kernels skip the leaf rows.  Up to three output sets receive the result
+// (the three-method call: the methods share u_res, hence the bonus token).
+struct NodeOutPtrs {
+    int32_t *accept_idx, *token, *hub;
+    float *beta, *rate;
+    uint32_t *status;
+};
+struct LeafArgs {
+    RowArgs r;
+    NodeOutPtrs out[3];
+    int n_out;
+};
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_leaf_kernel(LeafArgs A) {
+    __shared__ LeanShared sh;
+    const RowArgs &a = A.r;
+    const long long r = blockIdx.x;
+    const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
+    if (!(a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF)) return;
+    const __nv_bfloat16 *rowp = static_cast<const __nv_bfloat16 *>(a.target) + b * a.stride_seq + n * a.stride_node;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(rowp);
+    const Geo g = make_geo(a.vocab, 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lo = g.seg_lo(warp), hi = g.seg_hi(warp);
+    const float k = kLog2e / temperature_of(a, b);
+    const float ures = a.uniforms[r * 5 + 4];
+    const int CK = lean_ck_interval(g);
+    LeanAcc tp, unused;
+    unused.m2 = 0xff80ff80u; unused.s = 0.f; unused.c = 0.f;
+    lean_pass_a_ck(vp, lo, hi, lane, k, CK, tp, sh.cks[warp], sh.ckc[warp]);
+    ArgMaxSum Ps, unusedq;
+    lean_reduce2<false>(tp, unused, vp, vp, lo, hi, k, sh, Ps, unusedq);
+    const float Zp = Ps.sx + 1.f;
+    uint32_t status = 0;
+    int tok = -1;
+    if (!(Ps.ml > neg_inf()) || !(Ps.ml < -neg_inf()) || !finite_pos(Zp)) status = SPECHUB_ST_NONFINITE;
+    else tok = lean_ck_sample(g, rowp, k, Ps.c, CK, -1, ures, sh);
+    if (threadIdx.x == 0) {
+        for (int m = 0; m < A.n_out; ++m) {
+            const NodeOutPtrs &o = A.out[m];
+            o.accept_idx[r] = -1;
+            o.token[r] = tok;
+            if (o.hub) o.hub[r] = -1;
+            if (o.beta) { o.beta[2 * r] = 0.f; o.beta[2 * r + 1] = 0.f; }
+            if (o.rate) { o.rate[3 * r] = 0.f; o.rate[3 * r + 1] = 0.f; o.rate[3 * r + 2] = status ? 0.f : 1.f; }
+            if (o.status) o.status[r] = status;
+        }
+    }
+}
+
 // Passes B and C work on the exponentials themselves, in units of 1 / Z_p: with rho = Z_p / Z_q,
 //   d = e_p - rho e_q = Z_p (p - q),   t = max(d, 0) - s rho e_q = Z_p (max(p - q, 0) - s q),
 // two FMAs per vocabulary pair instead of two multiplications by 1/Z, a subtraction and an FMA.
@@ -585,7 +804,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     const float k = kLog2e / temperature_of(a, b);
     const float r1 = a.uniforms[r * 5 + 2], r2 = a.uniforms[r * 5 + 3], ures = a.uniforms[r * 5 + 4];
     const float pinf = -neg_inf();
-    const bool leaf = a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF;
+    // leaf rows of an unsplit call belong to lean_leaf_kernel
+    if (CS == 1 && a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF) return;
+    const bool leaf = CS > 1 && a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF;
     const bool writer = (me == 0 && threadIdx.x == 0);
 
     NodeResult o;
@@ -1002,170 +1223,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
 }
 
 // ------------------------------------------------------------------------------------------------
-// Draft step, one CTA per row, with a finer coarse CDF.  Pass A records, every CK lane-iterations,
-// the warp's sum since its previous checkpoint: sub-blocks of 32 * CK consecutive vectors, at most
-// kLeanCk per warp.  A draw then picks a sub-block from those sums and rescans only that (a few KB
-// instead of a warp's whole range), which is what the two-pass sampler costs most.
+// Draft step, one CTA per row (checkpointed pass A and sub-block sampler above).
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ int lean_ck_interval(const Geo &g) {
-    const int iters = (g.seg + 31) >> 5;
-    return 4 * max(1, (iters + 4 * kLeanCk - 1) / (4 * kLeanCk));   // a multiple of the unroll of pass A
-}
-
-__device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, int lane, float k, int CK,
-                                               LeanAcc &Q, float *cks, float *ckc) {
-    LeanAcc st;
-    st.m2 = 0xff80ff80u; st.s = 0.f; st.c = 0.f;
-    {   // one exponent reference for the whole warp: the maximum of its first vectors
-        float m0 = neg_inf();
-        if (lo + lane < hi) {
-            const uint4 a = rq[lo + lane];
-            m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m0 = fmaxf(m0, __shfl_xor_sync(kFull, m0, o));
-        if (m0 > neg_inf()) st.c = shift_of(m0, k);
-    }
-    float cref = st.c;              // the reference every lane is expected to hold
-    float tot = 0.f, ctot = st.c;   // this thread's sum over all checkpoints, on the scale ctot
-    int j = 0;
-    // checkpoint: the warp's sum since the last one.  A lane that had to move its reference (sums
-    // beyond 2^100, rare) is brought to the warp's largest reference first.
-    auto checkpoint = [&]() {
-        float contrib = st.s, cnow = cref;
-        if (__any_sync(kFull, st.c != cref)) {
-            float cm = st.c;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, o));
-            contrib = st.s > 0.f ? st.s * ex2(st.c - cm) : 0.f;
-            cnow = cm;
-        }
-        const float cs = warp_sum(contrib);
-        if (lane == 0) { cks[j] = cs; ckc[j] = cnow; }
-        ++j;
-        if (st.c != ctot) { tot = tot > 0.f ? tot * ex2(ctot - st.c) : 0.f; ctot = st.c; }
-        tot += st.s;
-        st.s = 0.f;
-    };
-    const int iters = (hi - lo + 31) >> 5;   // lane-iterations of this warp
-    const int nfull = (hi - lo) >> 5;        // those in which every lane has a vector
-    const uint4 *p = rq + lo + lane;
-    int it = 0, since = 0;
-    // four vectors per lane in flight; the next four are requested before the current ones are
-    // consumed, so that the checkpoint's shuffle chain overlaps the loads
-    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0, n3 = n0;
-    if (4 <= nfull) { n0 = p[0]; n1 = p[32]; n2 = p[64]; n3 = p[96]; }
-    for (; it + 4 <= nfull; it += 4) {
-        const uint4 a0 = n0, a1 = n1, a2 = n2, a3 = n3;
-        if (it + 8 <= nfull) {
-            n0 = p[32 * (it + 4)]; n1 = p[32 * (it + 5)]; n2 = p[32 * (it + 6)]; n3 = p[32 * (it + 7)];
-        }
-        lean_push(st, a0, k);
-        lean_push(st, a1, k);
-        lean_push(st, a2, k);
-        lean_push(st, a3, k);
-        since += 4;
-        if (since >= CK) { checkpoint(); since = 0; }
-    }
-    for (; it < iters; ++it) {
-        if (lo + lane + 32 * it < hi) lean_push(st, p[32 * it], k);
-        if (++since >= CK) { checkpoint(); since = 0; }
-    }
-    if (since > 0) checkpoint();
-    if (lane == 0)
-        for (; j < kLeanCk; ++j) { cks[j] = 0.f; ckc[j] = 0.f; }
-    Q.m2 = st.m2; Q.c = st.c; Q.s = tot;
-}
-
-// Inverse-CDF draw from softmax(row) without token `excl` (excl < 0: nothing left out) over the
-// checkpoint sub-blocks.  C = the row's exponent shift.  Returns to every thread the token, -1 if
-// nothing has mass.  Called by all threads of the CTA, after the checkpoints are visible.
-__device__ int lean_ck_sample(const Geo &g, const __nv_bfloat16 *row, float k, float C, int CK, int excl,
-                              float u, LeanShared &sh) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nslot = g.nwarps * kLeanCk;
-    auto wf = [&](int vi, float(&w)[8]) {
-        float v[8];
-        load_vec<__nv_bfloat16, true>(row, vi, g.V, v);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = (vi * 8 + i == excl) ? 0.f : ex2(__fmaf_rn(v[i], k, -C));
-    };
-    for (int s = threadIdx.x; s < nslot; s += blockDim.x) {
-        const float cs = sh.cks[s / kLeanCk][s % kLeanCk];
-        sh.ckm[s] = cs > 0.f ? cs * ex2(sh.ckc[s / kLeanCk][s % kLeanCk] - C) : 0.f;
-    }
-    __syncthreads();
-    if (excl >= 0) {
-        // the sub-block that holds the excluded token is summed again without it: subtracting the
-        // token's own term would cancel when that token carries most of the sub-block's mass
-        const int ev = excl >> 3;
-        const int w = g.warp_of_vec(ev), j = (ev - g.seg_lo(w)) / (32 * CK);
-        const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
-        float s = 0.f;
-        for (int vi = b0 + threadIdx.x; vi < b1; vi += blockDim.x) {
-            float wt[8];
-            wf(vi, wt);
-            s += ((wt[0] + wt[1]) + (wt[2] + wt[3])) + ((wt[4] + wt[5]) + (wt[6] + wt[7]));
-        }
-        s = warp_sum(s);
-        if (lane == 0) sh.mass[warp] = s;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float t = 0.f;
-            for (int x = 0; x < g.nwarps; ++x) t += sh.mass[x];
-            sh.ckm[w * kLeanCk + j] = t;
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x < 32) {   // warp 0: prefix sums over the sub-blocks, in id order
-        const int per = (nslot + 31) >> 5;
-        float ls = 0.f;
-        for (int i = 0; i < per; ++i) {
-            const int s = lane * per + i;
-            if (s < nslot) ls += sh.ckm[s];
-        }
-        float incl = ls;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float up = __shfl_up_sync(kFull, incl, o);
-            if (lane >= o) incl += up;
-        }
-        const float total = __shfl_sync(kFull, incl, 31);
-        const float t = u * total;
-        const unsigned pos = __ballot_sync(kFull, ls > 0.f);
-        const unsigned hit = __ballot_sync(kFull, ls > 0.f && incl > t);
-        if (!pos || !(total > 0.f)) {
-            if (lane == 0) sh.blk = -1;
-        } else {
-            const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
-            if (lane == L) {
-                float acc = incl - ls, lastacc = 0.f;
-                int sel = -1, last = -1;
-                for (int i = 0; i < per; ++i) {
-                    const int s = lane * per + i;
-                    const float m = s < nslot ? sh.ckm[s] : 0.f;
-                    if (m > 0.f) {
-                        last = s;
-                        lastacc = acc;
-                        if (sel < 0 && acc + m > t) { sel = s; sh.tt2 = t - acc; }
-                    }
-                    acc += m;
-                }
-                if (sel < 0) { sel = last; sh.tt2 = t - lastacc; }
-                sh.blk = sel;
-            }
-        }
-    }
-    __syncthreads();
-    const int slot = sh.blk;
-    const float tt = sh.tt2;
-    __syncthreads();   // range_sample3 reuses blk / tt2
-    if (slot < 0) return -1;
-    const int w = slot / kLeanCk, j = slot % kLeanCk;
-    const int b0 = g.seg_lo(w) + 32 * CK * j, b1 = min(g.seg_hi(w), b0 + 32 * CK);
-    return range_sample3(b0, b1, wf, sh, tt);
-}
-
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(RowArgs a, int method) {
     __shared__ LeanShared sh;
