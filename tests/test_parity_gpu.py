@@ -134,6 +134,26 @@ def test_lean_shapes(sh, V, split):
         sh.set_row_split(0)
 
 
+@pytest.mark.parametrize("V", [16384, 40000, 131072])
+def test_exponent_reference_moves(sh, V):
+    """Rows whose first logits lie hundreds of units below the later ones: the running sums leave
+    the range of their first exponent reference, in some lanes of a warp and not in others."""
+    rng = np.random.default_rng(V + 5)
+    B, N = 3, 7
+    lp, lq = random_logits(rng, B, N, V, "bf16")
+    lq[0, 0, : V // 2] -= 300.0; lp[0, 0, : V // 2] -= 300.0          # low first half, both rows
+    lq[0, 1, ::2] -= 250.0                                             # every other id low (lanes differ)
+    lp[0, 2, : V // 3] = -np.inf; lp[0, 2, V // 3: V // 2] -= 400.0    # -inf, then low, then normal
+    lq[1, 3, :100] += 300.0                                            # a high start, the rest far below
+    lq[1, 4, V - 50:] += 280.0; lp[1, 4, V - 50:] += 280.0             # the mass arrives at the very end
+    lq[2, 5, 1000:1010] += 200.0
+    lp, lq = workloads.round_to_storage(lp, "bf16"), workloads.round_to_storage(lq, "bf16")
+    un = random_uniforms(rng, B, N)
+    T = np.array([1.0, 0.7, 1.5], np.float32)
+    run_case(sh, lp, lq, "bf16", T, un, paper_layout=False, label="moving-reference")
+    run_case(sh, lp, lq, "bf16", 1.0, un, paper_layout=True, label="moving-reference-paper")
+
+
 @pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (12344, "bf16"), (40000, "bf16")])
 def test_decisions_without_probabilities(sh, V, dtype):
     """With no beta / rate buffers the library may stop after the first test; decisions, tokens,
