@@ -176,7 +176,10 @@ struct ArgMaxSum {
     float ml, c, sx;
     int idx;
     __device__ __forceinline__ void init() { ml = neg_inf(); c = 0.f; sx = 0.f; idx = 0x7fffffff; }
-    __device__ __forceinline__ float has() const { return ml > neg_inf() ? 1.f : 0.f; }
+    // The argmax's own term on this scale, 2^(k ml - c).  c is k*ml rounded to fp32, so this is
+    // 2^(rounding residual): 1 to within 1e-6 while |c| < 16, but 1 + 2e-5 at |c| = 500 (a large
+    // maximum logit or a small temperature); taking it as 1 would put that error into Z.
+    __device__ __forceinline__ float own(float k) const { return ml > neg_inf() ? ex2(fmaf(ml, k, -c)) : 0.f; }
 };
 template <int W>
 __device__ __forceinline__ void argmaxsum_push(ArgMaxSum &st, const float (&v)[W], int base, float k) {
@@ -189,7 +192,7 @@ __device__ __forceinline__ void argmaxsum_push(ArgMaxSum &st, const float (&v)[W
 #pragma unroll
         for (int i = W - 1; i >= 0; --i) pos = (v[i] == vmax) ? i : pos;
         const float cn = vmax * k;
-        st.sx = (st.sx + st.has()) * rescale(st.ml, st.c, cn);
+        st.sx = (st.sx + st.own(k)) * rescale(st.ml, st.c, cn);
         st.c = cn;
         st.ml = vmax;
         st.idx = base + pos;
@@ -201,15 +204,19 @@ __device__ __forceinline__ void argmaxsum_push(ArgMaxSum &st, const float (&v)[W
     }
     st.sx += acc;
 }
-__device__ __forceinline__ ArgMaxSum argmaxsum_merge(const ArgMaxSum &a, const ArgMaxSum &b) {
+// own term of a maximum logit ml on its own scale shift_of(ml, k)
+__device__ __forceinline__ float own_term(float ml, float k) {
+    return ml > neg_inf() ? ex2(fmaf(ml, k, -shift_of(ml, k))) : 0.f;
+}
+__device__ __forceinline__ ArgMaxSum argmaxsum_merge(const ArgMaxSum &a, const ArgMaxSum &b, float k) {
     const bool b_wins = (b.ml > a.ml) || (b.ml == a.ml && b.idx < a.idx);
     const ArgMaxSum &w = b_wins ? b : a;
     const ArgMaxSum &l = b_wins ? a : b;
     ArgMaxSum r = w;
-    r.sx = w.sx + (l.sx + l.has()) * rescale(l.ml, l.c, w.c);
+    r.sx = w.sx + (l.sx + l.own(k)) * rescale(l.ml, l.c, w.c);
     return r;
 }
-__device__ __forceinline__ ArgMaxSum argmaxsum_warp(ArgMaxSum st) {
+__device__ __forceinline__ ArgMaxSum argmaxsum_warp(ArgMaxSum st, float k) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         ArgMaxSum ot;
@@ -217,7 +224,7 @@ __device__ __forceinline__ ArgMaxSum argmaxsum_warp(ArgMaxSum st) {
         ot.c = __shfl_xor_sync(kFull, st.c, o);
         ot.sx = __shfl_xor_sync(kFull, st.sx, o);
         ot.idx = __shfl_xor_sync(kFull, st.idx, o);
-        st = argmaxsum_merge(st, ot);
+        st = argmaxsum_merge(st, ot, k);
     }
     return st;
 }

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     RowStat P, Q;
     merge_slices<1>(sh, 0, k, P);
     merge_slices<1>(sh, 1, k, Q);
-    const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
+    const float Zp = P.sx + P.own, Zq = Q.sx + Q.own;
     const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
     const float rho = __fdiv_rn(Zp, Zq);
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
@@ -113,9 +113,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     if (!ok_r[0]) o[1].status = SPECHUB_ST_TOKEN_RANGE;
     if (!ok_r[1]) o[2].status = SPECHUB_ST_TOKEN_RANGE;
     const bool degenerate = !(Q.sx > 0.f);
-    const float c = degenerate ? 0.f : 1.f / Q.sx;
+    const float c = degenerate ? 0.f : Q.own / Q.sx;
     const float crho = c * rho;
-    const float qa = invZq, rest = Q.sx * invZq;
+    const float qa = Q.own * invZq, rest = Q.sx * invZq;
     const int hubvec = hubtok >> 3, hubel = hubtok & 7;
     const int wx1 = ok_r[1] ? rx1[1] : -1;            // RRSw's first draft (left out of its renormaliser)
     const int wvec = wx1 >> 3, wel = wx1 & 7;
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
     __syncthreads();
     RowStat Q;
     merge_slices<1>(sh, 0, k, Q);
-    const float Zq = Q.sx + 1.f;
+    const float Zq = Q.sx + Q.own;
     if (!(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf())) {
         if (t0) {
             for (int m = 0; m < 3; ++m) {
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
     uint32_t st[3] = {0, 0, 0};
     int x2[3];
     // SpecHub (Section 4)
-    const float prob0 = 1.f / Zq;
+    const float prob0 = Q.own / Zq;
     float prob1 = 0.f;
     if (x1 != hubtok) {
         x2[0] = hubtok;

@@ -56,7 +56,7 @@ __device__ int sample_row_multi(const Geo &g, const LT *row, float k, float cQ, 
         const int w = threadIdx.x;
         const float ml = wp.ml[w];
         const bool holds_hub = (wp.idx[w] == hubtok);
-        const float own = (ml > neg_inf() && !(holds_hub && hub_out)) ? 1.f : 0.f;
+        const float own = (holds_hub && hub_out) ? 0.f : own_term(ml, k);
         sh.mass[w] = (wp.sx[w] + own) * rescale(ml, shift_of(ml, k), cQ);
     }
     __syncthreads();
@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(512) kary_draft_kernel(KaryArgs A) {
     const float *un = a.uniforms + r * (2 * K + 1);
 
     const ArgMaxSum q = pass_a<LT, AL>(g, rowq, k, sh.q);
-    const float Zq = q.sx + 1.f;
+    const float Zq = q.sx + q.own(k);
     uint32_t st = 0;
     int x[kMaxK];
     for (int i = 0; i < K; ++i) x[i] = -1;
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(512) kary_verify_kernel(KaryArgs A) {
     };
 
     const ArgMaxSum P = pass_a<LT, AL>(g, rowp, k, sh.p);
-    const float Zp = P.sx + 1.f;
+    const float Zp = P.sx + P.own(k);
     if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) { status = SPECHUB_ST_NONFINITE; write_out(); return; }
     const float cP = P.c, invZp = 1.f / Zp;
     if (a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF) {
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(512) kary_verify_kernel(KaryArgs A) {
         return;
     }
     const ArgMaxSum Q = pass_a<LT, AL>(g, rowq, k, sh.q);
-    const float Zq = Q.sx + 1.f;
+    const float Zq = Q.sx + Q.own(k);
     if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) { status = SPECHUB_ST_NONFINITE; write_out(); return; }
     const float cQ = Q.c, invZq = 1.f / Zq;
     int x[kMaxK];

@@ -416,6 +416,7 @@ __device__ __forceinline__ int pick_part(const float *m, int n, float t, float &
 // What every CTA of a row knows about one of its rows after the slices were merged.
 struct RowStat {
     float ml, C, sx;  // row max logit, its shift, sum without the row argmax
+    float own;        // the row argmax's own term 2^(k ml - C) (1 up to the rounding of C)
     int idx;          // row argmax
 };
 
@@ -429,9 +430,9 @@ __device__ __forceinline__ void merge_slices(const LeanShared &sh, int r, float 
         const LeanShared *ps = RowGroup<CS>::peer(&sh, c);
         ArgMaxSum o;
         o.ml = ps->x_ml[r]; o.c = shift_of(o.ml, k); o.sx = ps->x_sx[r]; o.idx = ps->x_idx[r];
-        tot = argmaxsum_merge(tot, o);
+        tot = argmaxsum_merge(tot, o, k);
     }
-    st.ml = tot.ml; st.C = tot.c; st.sx = tot.sx; st.idx = tot.idx;
+    st.ml = tot.ml; st.C = tot.c; st.sx = tot.sx; st.idx = tot.idx; st.own = tot.own(k);
 }
 
 // Mass of slice c of a row (row scale) for a draw from softmax(row) without token `excl`
@@ -442,7 +443,7 @@ __device__ __forceinline__ float slice_mass(const LeanShared &sh, int r, const R
                                             float k) {
     const LeanShared *ps = RowGroup<CS>::peer(&sh, c);
     const float ml = ps->x_ml[r];
-    const float own = (ml > neg_inf() && ps->x_idx[r] != excl) ? 1.f : 0.f;
+    const float own = (ps->x_idx[r] != excl) ? own_term(ml, k) : 0.f;
     return (ps->x_sx[r] + own) * rescale(ml, shift_of(ml, k), st.C);
 }
 
@@ -460,7 +461,7 @@ __device__ int lean_sample_slice(const Geo &g, const __nv_bfloat16 *row, float k
         const int w = threadIdx.x;
         const int lv = locarg >> 3;
         const bool holds = lml > neg_inf() && lv >= g.seg_lo(w) && lv < g.seg_hi(w);
-        sh.mass[w] = (sh.wmass[r][w] + ((holds && excl != locarg) ? 1.f : 0.f)) * f;
+        sh.mass[w] = (sh.wmass[r][w] + ((holds && excl != locarg) ? own_term(lml, k) : 0.f)) * f;
     }
     __syncthreads();
     if (excl >= 0 && excl != locarg && g.holds_vec(excl >> 3)) {
@@ -755,7 +756,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_leaf_kernel(Leaf
     lean_pass_a_ck(vp, lo, hi, lane, k, CK, tp, sh.cks[warp], sh.ckc[warp]);
     ArgMaxSum Ps, unusedq;
     lean_reduce2<false>(tp, unused, vp, vp, lo, hi, k, sh, Ps, unusedq);
-    const float Zp = Ps.sx + 1.f;
+    const float Zp = Ps.sx + Ps.own(k);
     uint32_t status = 0;
     int tok = -1;
     if (!(Ps.ml > neg_inf()) || !(Ps.ml < -neg_inf()) || !finite_pos(Zp)) status = SPECHUB_ST_NONFINITE;
@@ -832,7 +833,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     RowStat P, Q;
     merge_slices<CS>(sh, 0, k, P);
     merge_slices<CS>(sh, 1, k, Q);
-    const float Zp = P.sx + 1.f, Zq = Q.sx + 1.f;
+    const float Zp = P.sx + P.own, Zq = Q.sx + Q.own;
     const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
     const float rho = __fdiv_rn(Zp, Zq);
     const int x1 = a.draft_tokens_in[2 * r], x2 = a.draft_tokens_in[2 * r + 1];
@@ -860,9 +861,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             const int x = pair_xa ? x1 : x2;
             if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
             const bool degenerate = !(Q.sx > 0.f);
-            const float c = degenerate ? 0.f : 1.f / Q.sx;
+            const float c = degenerate ? 0.f : Q.own / Q.sx;
             const float crho = c * rho;
-            const float qa = invZq, rest = Q.sx * invZq;
+            const float qa = Q.own * invZq, rest = Q.sx * invZq;
             const int hubvec = hubtok >> 3, hubel = hubtok & 7;
             const float px = prob_p(x), qx = prob_q(x);
             if (!a.beta && !a.rate) {
@@ -1132,7 +1133,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
     RowGroup<CS>::sync();  // [1]
     RowStat Q;
     merge_slices<CS>(sh, 0, k, Q);
-    const float Zq = Q.sx + 1.f;
+    const float Zq = Q.sx + Q.own;
     uint32_t st = 0;
     const bool bad = !(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf());
     const int hubtok = bad ? -1 : Q.idx;
@@ -1161,7 +1162,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
         bool x2_elsewhere = false;  // x2 (and its probability) written by the CTA that draws it
         int x2 = -1;
         if (method == kSpecHub) {
-            prob0 = 1.f / Zq;
+            prob0 = Q.own / Zq;
             if (x1 != hubtok) {
                 x2 = hubtok;
                 prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)) / Zq;
@@ -1250,7 +1251,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(
     __syncthreads();
     RowStat Q;
     merge_slices<1>(sh, 0, k, Q);
-    const float Zq = Q.sx + 1.f;
+    const float Zq = Q.sx + Q.own;
     uint32_t st = 0;
     int x1 = -1, x2 = -1, hubtok = -1;
     float prob0 = 0.f, prob1 = 0.f;
@@ -1260,7 +1261,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(
         hubtok = Q.idx;
         x1 = lean_ck_sample(g, rowq, k, Q.C, CK, -1, u1, sh);
         if (method == kSpecHub) {
-            prob0 = 1.f / Zq;
+            prob0 = Q.own / Zq;
             if (x1 != hubtok) {
                 x2 = hubtok;
                 prob1 = ex2(fmaf(load_one<__nv_bfloat16>(rowq, x1), k, -Q.C)) / Zq;

@@ -38,6 +38,7 @@ struct ShardArgs {
 
 struct ShardStat {
     float ml, C, sx;
+    float own;   // the row argmax's own term 2^(k ml - C)
     int idx;
 };
 
@@ -51,16 +52,16 @@ __device__ __forceinline__ ArgMaxSum shard_partial(const ShardArgs &a, int c, lo
 __device__ __forceinline__ ShardStat shard_merge(const ShardArgs &a, long long row, int which, float k) {
     ArgMaxSum tot;
     tot.init();
-    for (int c = 0; c < a.nranks; ++c) tot = argmaxsum_merge(tot, shard_partial(a, c, row, which, k));
+    for (int c = 0; c < a.nranks; ++c) tot = argmaxsum_merge(tot, shard_partial(a, c, row, which, k), k);
     ShardStat st;
-    st.ml = tot.ml; st.C = tot.c; st.sx = tot.sx; st.idx = tot.idx;
+    st.ml = tot.ml; st.C = tot.c; st.sx = tot.sx; st.idx = tot.idx; st.own = tot.own(k);
     return st;
 }
 // Mass of rank c's slice in a draw from softmax(row) without token excl, on the row's scale.
 __device__ __forceinline__ float shard_mass(const ShardArgs &a, int c, long long row, int which, float k,
                                             const ShardStat &st, int excl) {
     const ArgMaxSum o = shard_partial(a, c, row, which, k);
-    const float own = (o.ml > neg_inf() && o.idx != excl) ? 1.f : 0.f;
+    const float own = (o.idx != excl) ? o.own(k) : 0.f;
     return (o.sx + own) * rescale(o.ml, o.c, st.C);
 }
 
@@ -120,7 +121,7 @@ __device__ __forceinline__ ShardRow shard_row(const ShardArgs &a) {
     return w;
 }
 __device__ __forceinline__ bool shard_bad(const ShardStat &s) {
-    return !(s.ml > neg_inf()) || !(s.ml < -neg_inf()) || !finite_pos(s.sx + 1.f);
+    return !(s.ml > neg_inf()) || !(s.ml < -neg_inf()) || !finite_pos(s.sx + s.own);
 }
 
 // ---- phase "stats" ------------------------------------------------------------------------------
@@ -162,11 +163,11 @@ __device__ __forceinline__ ShardPair shard_pair(const ShardArgs &a, const ShardR
     ShardPair s;
     s.P = shard_merge(a, w.r, 0, w.k);
     s.Q = shard_merge(a, w.r, 1, w.k);
-    s.invZp = 1.f / (s.P.sx + 1.f);
-    s.invZq = 1.f / (s.Q.sx + 1.f);
+    s.invZp = 1.f / (s.P.sx + s.P.own);
+    s.invZq = 1.f / (s.Q.sx + s.Q.own);
     s.hub = s.Q.idx;
     s.degenerate = !(s.Q.sx > 0.f);
-    s.c = s.degenerate ? 0.f : 1.f / s.Q.sx;
+    s.c = s.degenerate ? 0.f : s.Q.own / s.Q.sx;
     const int x1 = a.r.draft_tokens_in[2 * w.r], x2 = a.r.draft_tokens_in[2 * w.r + 1];
     s.pair_xa = (x2 == s.hub && x1 != s.hub);
     const bool pair_ax = (x1 == s.hub && x2 != s.hub);
@@ -264,7 +265,7 @@ __global__ void __launch_bounds__(512) shard_decide_kernel(ShardArgs a) {
 #pragma unroll
             for (int i = 0; i < 6; ++i) tot[i] += gs[i];
         }
-        const float qa = s.invZq, rest = s.Q.sx * s.invZq;
+        const float qa = s.Q.own * s.invZq, rest = s.Q.sx * s.invZq;
         const float S1 = tot[0], S2 = s.degenerate ? qa : tot[1], R = tot[2];
         const float px = tot[3], qx = tot[4], pa = tot[5];
         const float hub_left = fmaxf(pa - S2, 0.f);

@@ -23,8 +23,8 @@ __device__ __forceinline__ RrsRow rrs_row(const ShardArgs &a, const ShardRow &w)
     RrsRow s;
     s.P = shard_merge(a, w.r, 0, w.k);
     s.Q = shard_merge(a, w.r, 1, w.k);
-    s.invZp = 1.f / (s.P.sx + 1.f);
-    s.invZq = 1.f / (s.Q.sx + 1.f);
+    s.invZp = 1.f / (s.P.sx + s.P.own);
+    s.invZq = 1.f / (s.Q.sx + s.Q.own);
     s.x1 = a.r.draft_tokens_in[2 * w.r];
     s.x2 = a.r.draft_tokens_in[2 * w.r + 1];
     s.ok = s.x1 >= 0 && s.x1 < a.vocab_total && s.x2 >= 0 && s.x2 < a.vocab_total;

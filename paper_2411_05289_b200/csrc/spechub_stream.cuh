@@ -63,7 +63,7 @@ __device__ ArgMaxSum pass_a(const Geo &g, const LT *row, float k, WarpPart &wp) 
         load_vec<LT, AL>(row, vi, g.V, v);
         argmaxsum_push<VW>(st, v, vi * VW, k);
     }
-    st = argmaxsum_warp(st);
+    st = argmaxsum_warp(st, k);
     if (lane == 0) { wp.ml[warp] = st.ml; wp.sx[warp] = st.sx; wp.idx[warp] = st.idx; }
     __syncthreads();
     ArgMaxSum tot;
@@ -71,7 +71,7 @@ __device__ ArgMaxSum pass_a(const Geo &g, const LT *row, float k, WarpPart &wp) 
     for (int w = 0; w < g.nwarps; ++w) {
         ArgMaxSum o;
         o.ml = wp.ml[w]; o.c = shift_of(o.ml, k); o.sx = wp.sx[w]; o.idx = wp.idx[w];
-        tot = argmaxsum_merge(tot, o);
+        tot = argmaxsum_merge(tot, o, k);
     }
     return tot;
 }
@@ -102,7 +102,7 @@ __device__ int sample_row(const Geo &g, const LT *row, float k, float cQ, int hu
         const float ml = wp.ml[w];
         const bool holds_hub = (wp.idx[w] == hubtok);
         // the warp's partial leaves out its own argmax: add it back unless it is the excluded hub
-        const float own = (ml > neg_inf() && !(holds_hub && excl == hubtok)) ? 1.f : 0.f;
+        const float own = (holds_hub && excl == hubtok) ? 0.f : own_term(ml, k);
         sh.mass[w] = (wp.sx[w] + own) * rescale(ml, shift_of(ml, k), cQ);
     }
     __syncthreads();
@@ -146,7 +146,8 @@ __global__ void __launch_bounds__(512) draft_rows_kernel(RowArgs a, int method) 
     const float u1 = a.uniforms[r * 5 + 0], u2 = a.uniforms[r * 5 + 1];
 
     const ArgMaxSum q = pass_a<LT, AL>(g, rowq, k, sh.q);
-    const float Zq = q.sx + 1.f;
+    const float eq_a = q.own(k);   // the hub's own term, 2^(k l(a) - c)
+    const float Zq = q.sx + eq_a;
     uint32_t st = 0;
     int x1 = -1, x2 = -1, hubtok = -1;
     float prob0 = 0.f, prob1 = 0.f;
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(512) draft_rows_kernel(RowArgs a, int method) 
         hubtok = q.idx;
         x1 = sample_row<LT, AL>(g, rowq, k, q.c, hubtok, -1, u1, sh.q, sh);
         if (method == kSpecHub) {
-            prob0 = 1.f / Zq;
+            prob0 = eq_a / Zq;
             if (x1 != hubtok) {
                 x2 = hubtok;
                 prob1 = ex2(fmaf(load_one<LT>(rowq, x1), k, -q.c)) / Zq;
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(512) verify_rows_kernel(RowArgs a) {
     o.beta[0] = o.beta[1] = 0.f; o.rate[0] = o.rate[1] = o.rate[2] = 0.f;
 
     const ArgMaxSum P = pass_a<LT, AL>(g, rowp, k, sh.p);
-    const float Zp = P.sx + 1.f;
+    const float Zp = P.sx + P.own(k);
     if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) {
         o.status = SPECHUB_ST_NONFINITE;
         if (threadIdx.x == 0) write_node(a, r, o);
@@ -269,7 +270,8 @@ __global__ void __launch_bounds__(512) verify_rows_kernel(RowArgs a) {
     }
 
     const ArgMaxSum Q = pass_a<LT, AL>(g, rowq, k, sh.q);
-    const float Zq = Q.sx + 1.f;
+    const float eq_a = Q.own(k);   // the hub's own term, 2^(k l(a) - c)
+    const float Zq = Q.sx + eq_a;
     if (!(Q.ml > neg_inf()) || !(Q.ml < pinf) || !finite_pos(Zq)) {
         o.status = SPECHUB_ST_NONFINITE;
         if (threadIdx.x == 0) write_node(a, r, o);
@@ -291,8 +293,8 @@ __global__ void __launch_bounds__(512) verify_rows_kernel(RowArgs a) {
             return;
         }
         const bool degenerate = !(Q.sx > 0.f);           // 1 - q(a) = 0
-        const float c = degenerate ? 0.f : 1.f / Q.sx;     // q(a) / (1 - q(a))
-        const float qa = invZq, rest = Q.sx * invZq;
+        const float c = degenerate ? 0.f : eq_a / Q.sx;    // q(a) / (1 - q(a))
+        const float qa = eq_a * invZq, rest = Q.sx * invZq;
         if (!a.beta && !a.rate) {
             // No probability is asked for: the first test needs scalars only, and if it accepts the
             // transport sums decide nothing.
