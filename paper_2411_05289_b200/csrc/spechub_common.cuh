@@ -192,7 +192,7 @@ __device__ __forceinline__ void argmaxsum_push(ArgMaxSum &st, const float (&v)[W
 #pragma unroll
         for (int i = W - 1; i >= 0; --i) pos = (v[i] == vmax) ? i : pos;
         const float cn = vmax * k;
-        st.sx = (st.sx + st.own(k)) * rescale(st.ml, st.c, cn);
+        st.sx = __fmul_rn(__fadd_rn(st.sx, st.own(k)), rescale(st.ml, st.c, cn));
         st.c = cn;
         st.ml = vmax;
         st.idx = base + pos;
@@ -213,7 +213,9 @@ __device__ __forceinline__ ArgMaxSum argmaxsum_merge(const ArgMaxSum &a, const A
     const ArgMaxSum &w = b_wins ? b : a;
     const ArgMaxSum &l = b_wins ? a : b;
     ArgMaxSum r = w;
-    r.sx = w.sx + (l.sx + l.own(k)) * rescale(l.ml, l.c, w.c);
+    // roundings pinned (no contraction into an FMA): the target and the draft row go through separately
+    // inlined copies of this code and must give the same bits when the rows are equal
+    r.sx = __fadd_rn(w.sx, __fmul_rn(__fadd_rn(l.sx, l.own(k)), rescale(l.ml, l.c, w.c)));
     return r;
 }
 __device__ __forceinline__ ArgMaxSum argmaxsum_warp(ArgMaxSum st, float k) {
