@@ -126,7 +126,9 @@ struct MaxSum {
     float ml, c, s;
     __device__ __forceinline__ void init() { ml = neg_inf(); c = 0.f; s = 0.f; }
 };
-__device__ __forceinline__ float shift_of(float ml, float k) { return ml > neg_inf() ? ml * k : 0.f; }
+// (the product is rounded on its own: were it contracted into a later subtraction, two copies of the
+// same code could disagree in the last bit)
+__device__ __forceinline__ float shift_of(float ml, float k) { return ml > neg_inf() ? __fmul_rn(ml, k) : 0.f; }
 // 2^(c_from - c_to) for a partial whose maximum is ml_from; an empty partial (no finite
 // logit yet) carries no mass, whatever the target shift is.
 __device__ __forceinline__ float rescale(float ml_from, float c_from, float c_to) {
@@ -139,7 +141,7 @@ __device__ __forceinline__ void maxsum_push(MaxSum &st, const float (&v)[W], flo
 #pragma unroll
     for (int i = 1; i < W; ++i) vmax = fmaxf(vmax, v[i]);
     if (vmax > st.ml) {
-        const float cn = vmax * k;
+        const float cn = __fmul_rn(vmax, k);
         st.s *= rescale(st.ml, st.c, cn);
         st.c = cn;
         st.ml = vmax;
@@ -191,7 +193,7 @@ __device__ __forceinline__ void argmaxsum_push(ArgMaxSum &st, const float (&v)[W
         int pos = 0;
 #pragma unroll
         for (int i = W - 1; i >= 0; --i) pos = (v[i] == vmax) ? i : pos;
-        const float cn = vmax * k;
+        const float cn = __fmul_rn(vmax, k);
         st.sx = __fmul_rn(__fadd_rn(st.sx, st.own(k)), rescale(st.ml, st.c, cn));
         st.c = cn;
         st.ml = vmax;
