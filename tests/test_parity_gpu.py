@@ -134,6 +134,23 @@ def test_lean_shapes(sh, V, split):
         sh.set_row_split(0)
 
 
+@pytest.mark.parametrize("V,dtype", [(1000, "fp32"), (12344, "bf16"), (40000, "bf16")])
+def test_low_temperature_large_logits(sh, V, dtype):
+    """Maximum logits of 20-40 at T = 0.05-0.3: k * max logit reaches several hundred, where the
+    rounding of that product is 1e-5 and may not leak into the normaliser."""
+    rng = np.random.default_rng(V + 77)
+    B, N = 4, 7
+    lp = rng.normal(0, 4.0, (B, N, V)).astype(np.float32) + 15.0
+    lq = lp + rng.normal(0, 0.3, (B, N, V)).astype(np.float32)
+    lp[:, :, 11] += 12.0; lq[:, :, 11] += 12.0        # a clear top token around 40
+    lp[:, :, 500] += 11.5; lq[:, :, 500] += 11.0
+    lp, lq = workloads.round_to_storage(lp, dtype), workloads.round_to_storage(lq, dtype)
+    un = random_uniforms(rng, B, N)
+    T = np.array([0.05, 0.1, 0.3, 1.0], np.float32)
+    run_case(sh, lp, lq, dtype, T, un, paper_layout=False, label="low-T")
+    run_case(sh, lp, lq, dtype, 0.1, un, paper_layout=True, label="low-T-paper")
+
+
 @pytest.mark.parametrize("V", [16384, 40000, 131072])
 def test_exponent_reference_moves(sh, V):
     """Rows whose first logits lie hundreds of units below the later ones: the running sums leave
