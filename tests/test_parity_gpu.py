@@ -493,3 +493,35 @@ def test_very_many_rows(sh):
         w = oracle.walk(out["accept_idx"], out["token"], 1)
         for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
             np.testing.assert_array_equal(out[k], w[k], err_msg="many-rows walk %s" % k)
+
+
+def test_calls_on_two_streams_do_not_interfere(sh):
+    """The library keeps no state: calls enqueued on two streams, interleaved, give what the same
+    calls give one after another."""
+    rng = np.random.default_rng(21)
+    cases = []
+    for V, dtype in ((12344, "bf16"), (5000, "fp32")):
+        lp, lq = random_logits(rng, 6, 7, V, dtype)
+        un = random_uniforms(rng, 6, 7)
+        cases.append((workloads.to_device(lp, dtype), workloads.to_device(lq, dtype), torch.from_numpy(un).cuda()))
+    tree = sh.Tree.heap(7)
+    ref = []
+    for tp, tq, und in cases:
+        d = sh.spechub_draft_sample(tq, und, tree, 1.0)
+        ref.append((d, sh.spechub_verify_tree(tp, tq, d["tokens"], und, tree, 1.0)))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    got = [None, None]
+    for rep in range(3):
+        for i, (tp, tq, und) in enumerate(cases):
+            with torch.cuda.stream(streams[i]):
+                d = sh.spechub_draft_sample(tq, und, tree, 1.0)
+                got[i] = (d, sh.spechub_verify_tree(tp, tq, d["tokens"], und, tree, 1.0))
+    torch.cuda.synchronize()
+    for (dr, vr), (dg, vg) in zip(ref, got):
+        assert torch.equal(dr["tokens"], dg["tokens"])
+        for k in vr:
+            a, b = vr[k], vg[k]
+            if a.dtype == torch.float32:
+                a, b = a.view(torch.int32), b.view(torch.int32)
+            assert torch.equal(a, b), k
