@@ -466,7 +466,10 @@ def main():
                     "steps": args.e2e_steps, "chunks": n_chunks,
                     "note": "pinned host buffers -> device -> public API -> pinned host results; "
                             "chunks of whole sequences on two streams (copies overlap kernels)"},
-            "gpu_launches": 9 * args.steps,
+            # per step and method: draft kernel, verification kernel, walk kernel; in paper layout the
+            # large-vocabulary bf16 path adds a kernel for the leaf rows
+            "gpu_launches": (9 + (3 if args.layout == "paper" and cfg.dtype == "bf16" and cfg.vocab >= 8192
+                                  and cfg.vocab % 8 == 0 else 0)) * args.steps,
             "clocks": clocks,
             "roofline": roof["spechub_verify_tree"],
             "kernels": roof,
