@@ -177,6 +177,34 @@ class Tree:
             kind = kind.to(device)
         return Tree(levels=levels, child=None, node_kind=kind, k=k)
 
+    @staticmethod
+    def from_parents(parents, k: int = 2, leaves_sample: bool = True, device="cuda") -> "Tree":
+        """Any tree in level order from its parent list (``parents[0] = -1``; every parent index is
+        smaller than its child's; at most ``k`` children per node, in the order they are listed):
+        unbalanced trees such as the paper's binary Sequoia shapes.  Child slot i of a node is the
+        target of its draft i; missing children are -1.  With ``leaves_sample`` the childless
+        nodes only draw the bonus token from p."""
+        n = len(parents)
+        if n < 1 or parents[0] != -1:
+            raise ValueError("parents[0] must be -1 (the root)")
+        child = [[-1] * k for _ in range(n)]
+        depth = [1] * n
+        for c in range(1, n):
+            p = int(parents[c])
+            if not 0 <= p < c:
+                raise ValueError("node %d: parent %d must be an earlier node" % (c, p))
+            if depth[c - 1] > depth[p] + 1:
+                raise ValueError("nodes must be listed level by level")
+            slot = next((i for i in range(k) if child[p][i] < 0), None)
+            if slot is None:
+                raise ValueError("node %d has more than %d children" % (p, k))
+            child[p][slot] = c
+            depth[c] = depth[p] + 1
+        kind = None
+        if leaves_sample:
+            kind = torch.tensor([1 if all(x < 0 for x in row) else 0 for row in child], dtype=torch.uint8).to(device)
+        return Tree(levels=max(depth), child=torch.tensor(child, dtype=torch.int32).to(device), node_kind=kind, k=k)
+
     def nodes_of_complete_tree(self) -> int:
         return (self.k ** self.levels - 1) // (self.k - 1)
 

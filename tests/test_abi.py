@@ -86,3 +86,21 @@ def test_product_path_does_not_reach_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower() or f == "__init__.py" and "oracle" not in text.lower(), f
+
+
+def test_tree_from_parents_builds_level_ordered_child_tables():
+    import numpy as np
+    import paper_2411_05289_b200 as sh
+
+    # an unbalanced binary tree: 0 -> (1, 2); 1 -> (3, 4); 2 -> (5); 3 -> (6)
+    t = sh.Tree.from_parents([-1, 0, 0, 1, 1, 2, 3], device="cpu")
+    assert t.levels == 4 and t.k == 2
+    np.testing.assert_array_equal(t.child.numpy(), [[1, 2], [3, 4], [5, -1], [6, -1], [-1, -1], [-1, -1], [-1, -1]])
+    np.testing.assert_array_equal(t.node_kind.numpy(), [0, 0, 0, 0, 1, 1, 1])
+    # the complete binary tree in heap order is the special case
+    h = sh.Tree.from_parents([-1] + [(c - 1) // 2 for c in range(1, 7)], leaves_sample=False, device="cpu")
+    np.testing.assert_array_equal(h.child.numpy()[:3], [[1, 2], [3, 4], [5, 6]])
+    assert h.node_kind is None and h.levels == 3
+    for bad in ([0, 0], [-1, 1], [-1, 0, 0, 0], [-1, 0, 0, 1, 3, 2]):
+        with pytest.raises(ValueError):
+            sh.Tree.from_parents(bad, device="cpu")

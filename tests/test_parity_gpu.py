@@ -525,3 +525,29 @@ def test_calls_on_two_streams_do_not_interfere(sh):
             if a.dtype == torch.float32:
                 a, b = a.view(torch.int32), b.view(torch.int32)
             assert torch.equal(a, b), k
+
+
+def test_unbalanced_tree_from_parents(sh):
+    """A binary tree with missing children (the shape of the paper's unbalanced Sequoia trees):
+    childless nodes draw the bonus token, the walk follows the child table."""
+    parents = [-1, 0, 0, 1, 1, 2, 3, 3, 4, 6]
+    tree = sh.Tree.from_parents(parents)
+    child = tree.child.cpu().numpy()
+    kind = tree.node_kind.cpu().numpy()
+    N = len(parents)
+    rng = np.random.default_rng(31)
+    for V, dtype in ((9000, "bf16"), (777, "fp32")):
+        B = 6
+        lp, lq = random_logits(rng, B, N, V, dtype, sigma=0.6)
+        un = random_uniforms(rng, B, N)
+        tp, tq, und = workloads.to_device(lp, dtype), workloads.to_device(lq, dtype), torch.from_numpy(un).cuda()
+        for m in METHODS:
+            d = parity.to_numpy(gpu_draft(sh, m, tq, und, tree, 1.0))
+            _, od = parity.check_draft(m, lq, 1.0, un, d, label="unbalanced")
+            tok = od["tokens"].copy()
+            out = parity.to_numpy(gpu_verify(sh, m, tp, tq, torch.from_numpy(tok).cuda(), und, tree, 1.0))
+            parity.check_verify(m, lp, lq, 1.0, tok, un, kind, out, label="unbalanced")
+            w = oracle.walk(out["accept_idx"], out["token"], tree.levels, child=child, node_kind=kind)
+            for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+                np.testing.assert_array_equal(out[k], w[k], err_msg="unbalanced walk %s" % k)
+            assert out["n_accepted"].max() >= 2
