@@ -153,15 +153,15 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
             lean_push(P, a, k);
             lean_push(Q, b, k);
         }
-        return;
-    }
+    } else {
 #pragma unroll 2
-    for (; vi < hi; vi += 32) {
-        const uint4 a = rp[vi];
-        uint4 b;
-        if (BOTH) b = rq[vi];
-        lean_push(P, a, k);
-        if (BOTH) lean_push(Q, b, k);
+        for (; vi < hi; vi += 32) {
+            const uint4 a = rp[vi];
+            uint4 b;
+            if (BOTH) b = rq[vi];
+            lean_push(P, a, k);
+            if (BOTH) lean_push(Q, b, k);
+        }
     }
 }
 
