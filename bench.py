@@ -39,12 +39,12 @@ METHODS = ("spechub", "rrs", "rrsw")
 # row count (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not
 # captured for the current kernels.
 TRAFFIC_PER_ROW = {
-    ("spechub_draft_sample", "c4"): 275213952.0 / 992,
-    ("spechub_verify_tree", "c4"): 946823584.0 / 992,
-    ("rrs_draft_sample[rrs]", "c4"): 281278008.0 / 992,
-    ("rrs_verify_tree[rrs]", "c4"): 1318844176.0 / 992,
-    ("rrs_draft_sample[rrsw]", "c4"): 279413776.0 / 992,
-    ("rrs_verify_tree[rrsw]", "c4"): 1336045672.0 / 992,
+    ("spechub_draft_sample", "c4"): 275031600.0 / 992,
+    ("spechub_verify_tree", "c4"): 941715280.0 / 992,
+    ("rrs_draft_sample[rrs]", "c4"): 278423376.0 / 992,
+    ("rrs_verify_tree[rrs]", "c4"): 1319892128.0 / 992,
+    ("rrs_draft_sample[rrsw]", "c4"): 279134568.0 / 992,
+    ("rrs_verify_tree[rrsw]", "c4"): 1330579352.0 / 992,
 }
 
 
