@@ -90,6 +90,10 @@ extern "C" {
 #define SPECHUB_FLAG_SPLIT_1 1u
 #define SPECHUB_FLAG_SPLIT_2 2u
 #define SPECHUB_FLAG_SPLIT_4 4u
+/* Verification with the exponentials resident on chip (tensor memory + shared memory): one read of the
+ * row pair from HBM instead of two.  Not combined with a split flag.  Applies to the same shapes as the
+ * large-vocabulary bf16 kernels, up to 262144 ids; other shapes ignore it. */
+#define SPECHUB_FLAG_RESIDENT 8u
 
 /* node kinds */
 #define SPECHUB_NODE_VERIFY 0 /* run the accept/reject tests on the node's two drafts         */

@@ -143,8 +143,11 @@ typedef struct {
     double margin[3];  /* |r1 - N1/D1|, |r2 - N2/D2| (inf if not performed), residual-draw margin */
     double cond[2];    /* conditioning of N/D for test 1 / test 2: (|N| + beta |D|) / D, where |.|
                           is the sum of the absolute values of the terms the quantity is formed
-                          from; a relative error eps in every p(y), q(y) moves N/D by at most
-                          eps * cond.  Used only by the parity checker to size its tolerance. */
+                          from, each weighted by the number of perturbed factors it has
+                          (Q(a,y) = q(a) q(y) / (1 - q(a)) has three, RRSw's q(y) / (1 - q(x1))
+                          two); a relative error eps in every p(y), q(y) moves N/D by at most
+                          eps * cond to first order.  Used only by the parity checker to size
+                          its tolerance. */
     int32_t accept_idx; /* 0 / 1 = accepted child, -1 = rejected (token is the residual draw)  */
     int32_t token;      /* emitted token of this node                                          */
     int32_t hub;        /* a (SpecHub) or -1                                                   */
@@ -275,7 +278,11 @@ void orc_spechub_verify(const double *p, const double *q, int V, int a, int x1, 
     for (int y = 0; y < V; ++y) {
         if (y == a) continue;
         if (Q1xa[y] > 0.0) nS1 += Qxa[y] + p[y];
-        if (Q1ax[y] > 0.0) nS2 += Qax[y] + (p1[y] > 0.0 ? p[y] + Qxa[y] : 0.0);
+#ifndef ORC_PLANT_COND_NS2   /* (the pins of cond[] build a copy with the term dropped and must then fail) */
+        if (Q1ax[y] > 0.0) nS2 += 3.0 * Qax[y] + (p1[y] > 0.0 ? p[y] + Qxa[y] : 0.0);
+#else
+        if (Q1ax[y] > 0.0) nS2 += 3.0 * Qax[y];
+#endif
         ns_add(&s1, Q1xa[y]);
         ns_add(&s2, Q1ax[y]);
         ns_add(&m1, dmin(p[y], Qxa[y]));       /* pi(x,a,x) */
@@ -298,7 +305,7 @@ void orc_spechub_verify(const double *p, const double *q, int V, int a, int x1, 
                                &out->margin[1], !acc, &out->status);
         if (!acc && acc2) { out->accept_idx = 1; out->token = a; acc = 1; }
     } else {
-        acc = accept_test(r1, p1[x], Qax[x], p[x] + Qxa[x], Qax[x], &out->beta[0], &out->cond[0],
+        acc = accept_test(r1, p1[x], Qax[x], p[x] + Qxa[x], 3.0 * Qax[x], &out->beta[0], &out->cond[0],
                           &out->margin[0], 1, &out->status);
         if (acc) { out->accept_idx = 1; out->token = x; }
         int acc2 = accept_test(r2, p[a], S2, p[a], nS2, &out->beta[1], &out->cond[1],
@@ -411,8 +418,13 @@ void orc_rrs_verify(const double *p, const double *q, int V, int x1, int x2, dou
     int acc2 = 0;
     if (A1 > 0.0) {
         /* p_1(x2) = max(p - q, 0)(x2) / A1: both its own subtraction and A1's terms enter */
+#ifndef ORC_PLANT_COND_NN    /* (as above: a planted mistake for the pins of cond[]) */
         double nN = (p[x2] + q[x2]) / A1 + p1[x2] * nA1 / A1;
-        acc2 = accept_test(r2, p1[x2], q1[x2], nN, q1[x2], &out->beta[1], &out->cond[1],
+#else
+        double nN = (p[x2] + q[x2]) / A1;
+#endif
+        acc2 = accept_test(r2, p1[x2], q1[x2], nN, (without_replacement ? 2.0 : 1.0) * q1[x2], &out->beta[1],
+                           &out->cond[1],
                            &out->margin[1], !acc, &out->status);
     } else {
         out->beta[1] = 0.0;

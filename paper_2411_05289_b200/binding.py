@@ -135,10 +135,11 @@ _split = 0
 
 
 def set_row_split(ctas: int) -> None:
-    """Force 1, 2 or 4 CTAs per row in the large-vocabulary kernels (0 restores the default)."""
+    """Force 1, 2 or 4 CTAs per row in the large-vocabulary streaming kernels (0 restores the
+    default); 8 selects verification with the exponentials resident on chip (SPECHUB_FLAG_RESIDENT)."""
     global _split
-    if ctas not in (0, 1, 2, 4):
-        raise ValueError("row split must be 0, 1, 2 or 4")
+    if ctas not in (0, 1, 2, 4, 8):
+        raise ValueError("row split must be 0, 1, 2, 4 or 8 (8 = resident)")
     _split = ctas
 
 
@@ -218,6 +219,17 @@ def _stream_ptr(stream):
     return ctypes.c_void_p(s.cuda_stream)
 
 
+def _hold(tensors, stream):
+    """Temporaries of a call (a converted temperature vector, a workspace) are freed when the Python
+    call returns, while the kernels may still be queued.  On the current stream torch's allocator
+    orders the reuse after them; on any other stream it has to be told."""
+    if stream is None:
+        return
+    for t in tensors:
+        if t is not None:
+            t.record_stream(stream)
+
+
 def _desc(logits: torch.Tensor, tree: Tree, temperature) -> tuple:
     if logits.dim() != 3 or logits.stride(2) != 1:
         raise ValueError("logits must be [batch][nodes][vocab] with a contiguous vocabulary axis")
@@ -291,6 +303,7 @@ def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, st
     status = torch.empty((B, N), dtype=torch.int32, device=dev)
     _check(lib.spechub_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), _ptr(tokens),
                                     _ptr(hub), _ptr(prob), _ptr(status), _stream_ptr(stream)))
+    _hold(keep + [tokens, hub, prob, status], stream)
     return dict(tokens=tokens, hub=hub, prob=prob, status=status)
 
 
@@ -307,6 +320,7 @@ def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bo
     _check(lib.rrs_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
                                 int(bool(without_replacement)), _ptr(tokens), _ptr(status),
                                 _stream_ptr(stream)))
+    _hold(keep + [tokens, status], stream)
     return dict(tokens=tokens, status=status)
 
 
@@ -352,6 +366,7 @@ def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, t
         _check(lib.spechub_verify_tree(*common, *tail))
     else:
         _check(lib.rrs_verify_tree(*common, 1 if method == "rrsw" else 0, *tail))
+    _hold(keep + [ws] + list(out.values()), stream)
     return out
 
 
@@ -392,6 +407,7 @@ def mdsd_compare_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.
     sp = (ctypes.c_void_p * 3)(*[t.data_ptr() for t in status])
     _check(lib.mdsd_compare_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), tp, _ptr(hub),
                                          _ptr(prob), sp, _stream_ptr(stream)))
+    _hold(keep + tokens + status + [hub, prob], stream)
     return dict(spechub=dict(tokens=tokens[0], hub=hub, prob=prob, status=status[0]),
                 rrs=dict(tokens=tokens[1], status=status[1]),
                 rrsw=dict(tokens=tokens[2], status=status[2]))
@@ -426,6 +442,7 @@ def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
     _check(lib.mdsd_compare_verify_tree(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), tp,
                                         _ptr(uniforms), no, so, _ptr(ws), ws_bytes, _stream_ptr(stream)))
+    _hold(keep + [ws] + [t for m in METHODS for t in out[m].values()], stream)
     return out
 
 
@@ -457,6 +474,7 @@ def spechub_verify_tree_static(target_logits, draft_logits, draft_tokens, unifor
     _check(lib.spechub_verify_tree_static(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits),
                                           _ptr(draft_tokens), _ptr(uniforms), ctypes.byref(no),
                                           ctypes.byref(so), _stream_ptr(stream)))
+    _hold(keep + list(out.values()), stream)
     return out
 
 

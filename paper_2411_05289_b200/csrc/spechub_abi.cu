@@ -12,6 +12,7 @@
 #include "spechub_lean.cuh"
 #include "spechub_kary.cuh"
 #include "spechub_fused.cuh"
+#include "spechub_resident.cuh"
 #include "spechub_shard.cuh"
 #include "spechub_shard_rrs.cuh"
 
@@ -33,7 +34,8 @@ int check_desc(const spechub_desc *d) {
     if (!d->temperature_per_seq && !(d->temperature > 0.f && isfinite(d->temperature)))
         return SPECHUB_ERR_TEMPERATURE;
     const uint32_t split = d->flags & 7u;
-    if ((d->flags & ~7u) != 0 || (split & (split - 1)) != 0) return SPECHUB_ERR_SHAPE;
+    if ((d->flags & ~15u) != 0 || (split & (split - 1)) != 0) return SPECHUB_ERR_SHAPE;
+    if ((d->flags & SPECHUB_FLAG_RESIDENT) && split) return SPECHUB_ERR_SHAPE;
     if ((int64_t)d->batch * d->nodes > 0x7fffffffLL) return SPECHUB_ERR_SHAPE;
     return SPECHUB_OK;
 }
@@ -132,6 +134,84 @@ int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaS
 
 bool lean_ok(const spechub_desc *d, bool aligned) {
     return d->dtype == SPECHUB_BF16 && aligned && d->vocab % 8 == 0 && d->vocab >= 8192;
+}
+
+// ---- verification with the exponentials resident on chip ------------------------------------------
+// A row is spread over `cs` CTAs of 8 warps; every lane keeps `nb` batches of four 16-byte vectors
+// of the row pair as fp32 exponentials (tensor memory, shared memory, registers).  The smallest
+// cluster that holds the row with at most four batches per lane is taken.
+struct ResShape { int cs, nb; };
+
+bool resident_shape(const spechub_desc *d, bool aligned, ResShape *out) {
+    if (!lean_ok(d, aligned)) return false;
+    if (!(d->flags & SPECHUB_FLAG_RESIDENT)) return false;
+    const int nvec = d->vocab / 8;
+    for (int cs = 1; cs <= 8; cs *= 2) {
+        const int parts = cs * kResWarps;
+        const int seg = (((nvec + parts - 1) / parts) + 7) & ~7;   // vectors per warp, as the kernel cuts them
+        const int nb = (seg + 127) / 128;
+        if (nb <= kResMaxBatches) { out->cs = cs; out->nb = nb; return true; }
+    }
+    return false;
+}
+
+constexpr int kMaxDevices = 64;
+std::mutex g_attr_mutex;
+
+template <int MASK, int CS>
+int launch_resident_one(int nb, const FusedArgs &f, unsigned rows, cudaStream_t s) {
+    auto kern = resident_verify_kernel<MASK, CS>;
+    // tensor-memory columns of a CTA: two warps share each lane quarter, 32 columns per batch each
+    const uint32_t cols = nb == 1 ? 64u : nb == 2 ? 128u : 256u;
+    // Shared memory: e_q of all batches but the last.  A CTA that takes 256 columns asks for at least a
+    // third of an SM's shared memory, so that no more than two such CTAs share the SM's 512 columns.
+    int smem = (nb - 1) * 4 * 2 * kResThreads * 16;
+    if (cols == 256u && smem < 76 * 1024) smem = 76 * 1024;
+    constexpr int smem_max = (kResMaxBatches - 1) * 4 * 2 * kResThreads * 16;
+    static bool configured[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECHUB_ERR_LAUNCH;
+    {
+        std::lock_guard<std::mutex> lock(g_attr_mutex);
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) {
+                cudaGetLastError();
+                return SPECHUB_ERR_LAUNCH;
+            }
+            configured[dev] = true;
+        }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = CS > 1 ? 1 : 0;
+    cfg.gridDim = dim3(rows * CS); cfg.blockDim = dim3(kResThreads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    return cudaLaunchKernelEx(&cfg, kern, f, nb, cols) == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+}
+
+template <int MASK>
+int launch_resident_mask(ResShape sh, const FusedArgs &f, unsigned rows, cudaStream_t s) {
+    if (sh.cs == 1) return launch_resident_one<MASK, 1>(sh.nb, f, rows, s);
+    if (sh.cs == 2) return launch_resident_one<MASK, 2>(sh.nb, f, rows, s);
+    if (sh.cs == 4) return launch_resident_one<MASK, 4>(sh.nb, f, rows, s);
+    return launch_resident_one<MASK, 8>(sh.nb, f, rows, s);
+}
+
+// mask: bit m set = method m (0 SpecHub, 1 RRS, 2 RRSw) is verified; leaf rows go to lean_leaf_kernel
+int launch_resident(int mask, ResShape sh, const FusedArgs &f, unsigned rows, cudaStream_t s) {
+    if (f.r.node_kind) {
+        NodeOutPtrs outs[3];
+        int n_out = 0;
+        for (int m = 0; m < 3; ++m)
+            if (mask & (1 << m)) outs[n_out++] = f.out[m];
+        const int lrc = launch_lean_leaf(f.r, outs, n_out, rows, s);
+        if (lrc != SPECHUB_OK) return lrc;
+    }
+    if (mask == kMaskSpecHub) return launch_resident_mask<kMaskSpecHub>(sh, f, rows, s);
+    if (mask == kMaskRRS) return launch_resident_mask<kMaskRRS>(sh, f, rows, s);
+    if (mask == kMaskRRSw) return launch_resident_mask<kMaskRRSw>(sh, f, rows, s);
+    return launch_resident_mask<7>(sh, f, rows, s);
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH; }
@@ -252,6 +332,13 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
             if (al) kary_verify_kernel<float, true><<<rows, th, 0, s>>>(ka);
             else kary_verify_kernel<float, false><<<rows, th, 0, s>>>(ka);
         }
+    } else if (ResShape rs; resident_shape(d, al, &rs)) {
+        FusedArgs f = {};
+        f.r = a;
+        f.tok[method] = draft_tokens;
+        f.out[method] = NodeOutPtrs{a.accept_idx, a.token, a.hub, a.beta, a.rate, a.status};
+        const int lrc = launch_resident(1 << method, rs, f, rows, s);
+        if (lrc != SPECHUB_OK) return lrc;
     } else if (lean_ok(d, al)) {
         const int lrc = launch_lean_verify(method, lean_split(d), a, rows, s);
         if (lrc != SPECHUB_OK) return lrc;
@@ -328,12 +415,17 @@ int compare_verify(const spechub_desc *d, const void *target_logits, const void 
     }
     const unsigned rows = (unsigned)(d->batch * (int64_t)d->nodes);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (d->node_kind) {
-        const int llrc = launch_lean_leaf(f.r, f.out, 3, rows, s);
-        if (llrc != SPECHUB_OK) return llrc;
+    int lrc;
+    if (ResShape rs; resident_shape(d, al, &rs)) {
+        lrc = launch_resident(7, rs, f, rows, s);
+    } else {
+        if (d->node_kind) {
+            const int llrc = launch_lean_leaf(f.r, f.out, 3, rows, s);
+            if (llrc != SPECHUB_OK) return llrc;
+        }
+        fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
+        lrc = launch_status();
     }
-    fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
-    int lrc = launch_status();
     for (int m = 0; m < 3 && lrc == SPECHUB_OK && so; ++m) lrc = launch_walk(d, &no[m], &so[m], s);
     return lrc;
 }
@@ -617,7 +709,6 @@ static __device__ __align__(256) float g_static_scratch[(size_t)SPECHUB_STATIC_M
 
 namespace {
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 float *g_static_ptr[kMaxDevices] = {};
 

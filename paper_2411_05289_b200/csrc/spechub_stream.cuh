@@ -500,7 +500,7 @@ __global__ void walk_kernel(WalkArgs a) {
         ++emitted;
         if (a.node_kind && a.node_kind[n] == SPECHUB_NODE_LEAF) { ++step; break; }
         const int idx = a.accept_idx[r];
-        if (idx < 0) { ++step; break; }
+        if (idx < 0 || idx > 1) { ++step; break; }   // (a caller-supplied index outside {0, 1} ends the walk)
         ++acc;
         n = a.child ? a.child[2 * n + idx] : 2 * n + 1 + idx;
     }

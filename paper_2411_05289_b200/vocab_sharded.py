@@ -280,34 +280,47 @@ def shard_of_group(width: int, group=None) -> Shard:
     return Shard(r, n, sum(widths[:r]), sum(widths))
 
 
+def _on(stream):
+    """The drivers below mix kernel launches, allocations and collectives; all of them follow torch's
+    current stream, so a caller's stream is made current for the whole call (kernels launched on one
+    stream and collectives on another would race)."""
+    import contextlib
+
+    return contextlib.nullcontext() if stream is None else torch.cuda.stream(stream)
+
+
 def spechub_draft_sample_sharded(draft_slice, uniforms, tree, shard: Shard, temperature=1.0, group=None,
                                  stream=None):
-    d = ShardedDraft(draft_slice, uniforms, tree, shard, temperature, stream)
-    cand = d.candidates(all_gather_ranks(d.stats(), group))
-    return d.finish(all_max(cand, group))
+    with _on(stream):
+        d = ShardedDraft(draft_slice, uniforms, tree, shard, temperature, None)
+        cand = d.candidates(all_gather_ranks(d.stats(), group))
+        return d.finish(all_max(cand, group))
 
 
 def spechub_verify_tree_sharded(target_slice, draft_slice, draft_tokens, uniforms, tree, shard: Shard,
                                 temperature=1.0, group=None, stream=None):
-    v = ShardedVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, temperature, stream)
-    gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
-    return v.walk(all_max(v.decide(gsums), group))
+    with _on(stream):
+        v = ShardedVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, temperature, None)
+        gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
+        return v.walk(all_max(v.decide(gsums), group))
 
 
 def rrs_draft_sample_sharded(draft_slice, uniforms, tree, shard: Shard, without_replacement, temperature=1.0,
                              group=None, stream=None):
-    d = ShardedRrsDraft(draft_slice, uniforms, tree, shard, without_replacement, temperature, stream)
-    cand, ex1 = d.candidates(all_gather_ranks(d.stats(), group))
-    cand, ex1 = all_max(cand, group), all_max(ex1, group)
-    if without_replacement:
-        cand = all_max(d.second(cand, ex1), group)
-    return d.finish(cand)
+    with _on(stream):
+        d = ShardedRrsDraft(draft_slice, uniforms, tree, shard, without_replacement, temperature, None)
+        cand, ex1 = d.candidates(all_gather_ranks(d.stats(), group))
+        cand, ex1 = all_max(cand, group), all_max(ex1, group)
+        if without_replacement:
+            cand = all_max(d.second(cand, ex1), group)
+        return d.finish(cand)
 
 
 def rrs_verify_tree_sharded(target_slice, draft_slice, draft_tokens, uniforms, tree, shard: Shard,
                             without_replacement, temperature=1.0, group=None, stream=None):
-    v = ShardedRrsVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, without_replacement,
-                         temperature, stream)
-    gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
-    gw2 = all_gather_ranks(v.w2(gsums), group)
-    return v.walk(all_max(v.decide(gw2), group))
+    with _on(stream):
+        v = ShardedRrsVerify(target_slice, draft_slice, draft_tokens, uniforms, tree, shard, without_replacement,
+                             temperature, None)
+        gsums = all_gather_ranks(v.sums(all_gather_ranks(v.stats(), group)), group)
+        gw2 = all_gather_ranks(v.w2(gsums), group)
+        return v.walk(all_max(v.decide(gw2), group))
