@@ -59,8 +59,8 @@ struct __align__(16) ResShared {
     // per-part records, one slot per warp of the row, written by that warp into every CTA's copy
     float recA[kResMaxParts][12];  // c_p, s_p, c_q, s_q, max l_q, first id of the candidate hub logit,
                                    // s_q without exclusion candidate 0, 1, 2
-    float recB[kResMaxParts][4];   // S1, S2, R (SpecHub), A1 (RRS / RRSw)
-    float recC[kResMaxParts][4];   // W2 of RRS, W2 of RRSw
+    float recB[kResMaxParts][8];   // S1, S2, R (SpecHub), A1 (RRS / RRSw); R of each of the warp's batches
+    float recC[kResMaxParts][12];  // W2 of RRS, W2 of RRSw, -, -; W2 of RRS per batch; W2 of RRSw per batch
     int recH[kResMaxParts];        // first id of the row maximum (rows whose pair lacks the hub)
     float bc[24];                  // row values from warp 0 to the CTA
     int bi[12];
@@ -226,10 +226,13 @@ __device__ __forceinline__ float res_total(const V2 (&acc)[4]) {
 }
 
 // Inverse-CDF pick over the parts of a row (ascending token ranges), by one warp: lane l holds the
-// masses of parts 2l and 2l+1.  The first part with mass whose inclusive prefix exceeds t, else the
-// last part with mass; -1 when nothing has mass.  `base` = the mass before the picked part.
-__device__ __forceinline__ int res_pick(float m0, float m1, float t, int lane, float &base) {
-    const float ls = m0 + m1;
+// masses m[0..8) of eight consecutive parts (parts 8l .. 8l+7).  The first part with mass whose
+// inclusive prefix exceeds t, else the last part with mass; -1 when nothing has mass.  `base` = the
+// mass before the picked part.
+__device__ __forceinline__ int res_pick8(const float (&m)[8], float t, int lane, float &base) {
+    float ls = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ls += m[i];
     float incl = ls;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -237,20 +240,22 @@ __device__ __forceinline__ int res_pick(float m0, float m1, float t, int lane, f
         if (lane >= o) incl += up;
     }
     const float excl = incl - ls;
-    const unsigned pos = __ballot_sync(kFull, m0 > 0.f || m1 > 0.f);
-    const unsigned hit = __ballot_sync(kFull, (m0 > 0.f || m1 > 0.f) && incl > t);
+    const unsigned pos = __ballot_sync(kFull, ls > 0.f);
+    const unsigned hit = __ballot_sync(kFull, ls > 0.f && incl > t);
     if (!pos) { base = 0.f; return -1; }
     const int L = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));
-    int sel;
-    float bs;
-    if (hit) {
-        if (m0 > 0.f && excl + m0 > t) { sel = 2 * lane; bs = excl; }
-        else if (m1 > 0.f) { sel = 2 * lane + 1; bs = excl + m0; }
-        else { sel = 2 * lane; bs = excl; }
-    } else {
-        if (m1 > 0.f) { sel = 2 * lane + 1; bs = excl + m0; }
-        else { sel = 2 * lane; bs = excl; }
+    int sel = -1, last = -1;
+    float bs = 0.f, lastbs = 0.f, run = excl;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (m[i] > 0.f) {
+            last = 8 * lane + i;
+            lastbs = run;
+            if (sel < 0 && run + m[i] > t) { sel = last; bs = run; }
+        }
+        run += m[i];
     }
+    if (sel < 0) { sel = last; bs = lastbs; }
     base = __shfl_sync(kFull, bs, L);
     return __shfl_sync(kFull, sel, L);
 }
@@ -306,9 +311,13 @@ enum { kDrawP = 0, kDrawSpecHub = 1, kDrawAlg1 = 2 };
 // Verification: SpecHub (Algorithm 3 with the closed form of Section 4 / Appendix B.1), RRS and
 // RRSw (Algorithm 1), any subset of the three (MASK) on the same rows.  NB = batches per lane.
 // ------------------------------------------------------------------------------------------------
+struct ResRaw {   // one batch of a lane: four 16-byte vectors of each row, as loaded
+    uint4 p[4], q[4];
+};
+
 template <int MASK, int CS>
 __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedArgs A, int NB, uint32_t tmem_cols) {
-    constexpr int W = CS * kResWarps;   // parts (warps) per row
+    constexpr int W = CS * kResWarps;   // warps per row
     constexpr bool kSH = (MASK & kMaskSpecHub) != 0, kR = (MASK & kMaskRRS) != 0, kRW = (MASK & kMaskRRSw) != 0;
     constexpr bool kAlg1 = kR || kRW;
     extern __shared__ float4 eq_store[];   // e_q of the batches but the last: [slot][half][thread] as float4
@@ -330,23 +339,40 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
     const uint4 *vp = reinterpret_cast<const uint4 *>(rowp), *vq = reinterpret_cast<const uint4 *>(rowq);
     const int V = a.vocab, nvec = V >> 3;
     const int g = me * kResWarps + warp;
-    const int seg = (((nvec + W - 1) / W) + 7) & ~7;   // vectors per part (host: seg <= 128 NB)
+    const int seg = (((nvec + W - 1) / W) + 7) & ~7;   // vectors per warp (host: seg <= 128 NB)
     const int lo = min(g * seg, nvec), hi = min(lo + seg, nvec);
-    const float k = kLog2e / temperature_of(a, b);
-    const V2 k2 = v2_make(k, k);
     const bool writer = (me == 0 && threadIdx.x == 0);
     const int LB = NB - 1;   // the batch whose e_q stays in registers
 
-    // draft tokens of the methods and the logits at them (scalars every test needs)
+    // the draft tokens first: the logits at them are gathered below, behind the first vector loads
     int x1[3], x2[3];
     bool ok1[3], ok2[3];
+#pragma unroll
+    for (int m = 0; m < 3; ++m) {
+        x1[m] = x2[m] = -1;
+        if (MASK & (1 << m)) { x1[m] = A.tok[m][2 * r]; x2[m] = A.tok[m][2 * r + 1]; }
+    }
+    auto load_raw = [&](int bt, ResRaw &R) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int vi = lo + lane + 32 * (4 * bt + j);
+            R.p[j] = R.q[j] = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf
+            if (vi < hi) { R.p[j] = ld_stream(vp + vi); R.q[j] = ld_stream(vq + vi); }
+        }
+    };
+    ResRaw X, Y;   // two batches in flight: one is consumed while the other arrives
+    load_raw(0, X);
+    if (NB > 1) load_raw(1, Y);
+    else Y = X;
+
+    const float k = kLog2e / temperature_of(a, b);
+    const V2 k2 = v2_make(k, k);
     float lp1[3], lp2[3], lq1[3], lq2[3];
 #pragma unroll
     for (int m = 0; m < 3; ++m) {
-        x1[m] = x2[m] = -1; ok1[m] = ok2[m] = false;
+        ok1[m] = ok2[m] = false;
         lp1[m] = lp2[m] = lq1[m] = lq2[m] = 0.f;
         if (MASK & (1 << m)) {
-            x1[m] = A.tok[m][2 * r]; x2[m] = A.tok[m][2 * r + 1];
             ok1[m] = x1[m] >= 0 && x1[m] < V; ok2[m] = x2[m] >= 0 && x2[m] < V;
             const int i1 = ok1[m] ? x1[m] : 0, i2 = ok2[m] ? x2[m] : 0;
             if (warp == 0) {   // only warp 0 takes the decisions
@@ -379,7 +405,6 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
     // ---- storage --------------------------------------------------------------------------------------
     const uint32_t lane_field = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t col0 = static_cast<uint32_t>((warp >> 2) * (32 * NB));
-    float eqk[32];   // e_q of the last batch
     auto eq_ptr = [&](int slot) { return eq_store + (2 * slot) * kResThreads + threadIdx.x; };
     auto store_eq = [&](int slot, const float (&e)[8]) {
         float4 *dst = eq_ptr(slot);
@@ -427,23 +452,15 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
         }
         tmem_wait_st();
     };
-    // One batch: references, exponentials, stores, sums.  LAST: e_q goes to eqk instead of shared memory.
-    auto pass_a_batch = [&](int bt, auto last_tag) {
-        constexpr bool LAST = decltype(last_tag)::value;
-        uint4 rp[4], rq[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int vi = lo + lane + 32 * (4 * bt + j);
-            rp[j] = rq[j] = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf
-            if (vi < hi) { rp[j] = ld_stream(vp + vi); rq[j] = ld_stream(vq + vi); }
-        }
-        const float mpb = res_max4(rp), mqb = res_max4(rq);
+    // References of a batch, before its exponentials are taken.
+    auto batch_refs = [&](int bt, const ResRaw &R) {
+        const float mpb = res_max4(R.p), mqb = res_max4(R.q);
         mq_t = fmaxf(mq_t, mqb);
         if (kSH && mqb == Lc) {   // rare: this batch holds an id with the candidate hub logit
 #pragma unroll
             for (int j = 3; j >= 0; --j) {
                 float v[8];
-                unpack_bf16x8(rq[j], v);
+                unpack_bf16x8(R.q[j], v);
                 const int vi = lo + lane + 32 * (4 * bt + j);
 #pragma unroll
                 for (int i = 7; i >= 0; --i)
@@ -471,28 +488,58 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
                 if (mvq) c_qt = rqb;
             }
         }
+    };
+    // One batch but the last: exponentials to tensor / shared memory, sums.
+    auto pass_a_batch = [&](int bt, const ResRaw &R) {
+        batch_refs(bt, R);
         const V2 ncp2 = v2_make(-c_pt, -c_pt), ncq2 = v2_make(-c_qt, -c_qt);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             float e[8];
-            res_exp8(rp[j], k2, ncp2, e, pacc);
+            res_exp8(R.p[j], k2, ncp2, e, pacc);
             tmem_st8(taddr + 8 * (4 * bt + j), e);
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             float e[8];
-            res_exp8(rq[j], k2, ncq2, e, qacc);
-            if (LAST) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) eqk[8 * j + i] = e[i];
-            } else {
-                store_eq(4 * bt + j, e);
-            }
+            res_exp8(R.q[j], k2, ncq2, e, qacc);
+            store_eq(4 * bt + j, e);
         }
     };
+    // the next batch but one is requested as soon as a buffer is free
 #pragma unroll 1
-    for (int bt = 0; bt < LB; ++bt) pass_a_batch(bt, std::false_type{});
-    pass_a_batch(LB, std::true_type{});
+    for (int bt = 0; bt < LB; bt += 2) {
+        pass_a_batch(bt, X);
+        if (bt + 2 <= LB) load_raw(bt + 2, X);
+        if (bt + 1 < LB) {
+            pass_a_batch(bt + 1, Y);
+            if (bt + 3 <= LB) load_raw(bt + 3, Y);
+        }
+    }
+    float eqk[32];   // e_q of the last batch stays in registers
+    {
+        ResRaw L;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            L.p[j] = (LB & 1) ? Y.p[j] : X.p[j];
+            L.q[j] = (LB & 1) ? Y.q[j] : X.q[j];
+        }
+        batch_refs(LB, L);
+        const V2 ncp2 = v2_make(-c_pt, -c_pt), ncq2 = v2_make(-c_qt, -c_qt);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float e[8];
+            res_exp8(L.p[j], k2, ncp2, e, pacc);
+            tmem_st8(taddr + 8 * (4 * LB + j), e);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float e[8];
+            res_exp8(L.q[j], k2, ncq2, e, qacc);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) eqk[8 * j + i] = e[i];
+        }
+    }
     tmem_wait_st();
     const float sp_t = res_total(pacc), sq_t = res_total(qacc);
 
@@ -703,19 +750,30 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
     const float F = res_pow2(np), sc = res_pow2(nq - np);
     const float rho_t = __fmul_rn(rho_b, sc), crho_t = __fmul_rn(crho_b, sc);
     const V2 nrq2 = v2_make(-rho_t, -rho_t), nsq2 = v2_make(-crho_t, -crho_t);
-    // the slot of this lane that holds the hub / RRSw's first draft (-1: none)
+    // the slot of this lane that holds the hub (-1: none)
     const int hub_slot = (kSH && hubc >= 0) ? cslot[hubc] : -1;
     const bool hub_warp = kSH && hubc >= 0 && cwarp[hubc];
     const int hub_el = (kSH && hubc >= 0) ? (cand[hubc] & 7) : 0;
+    // a per-batch partial of this warp, to every CTA of the row
+    auto push_scalar = [&](float *slot, float v) {
+        if (lane < CS) {
+            float *dst = slot;
+            if (CS > 1) dst = cooperative_groups::this_cluster().map_shared_rank(slot, lane);
+            *dst = v;
+        }
+    };
 
     // ---- pass B over the stored exponentials: S1, S2, R (ids != a) and A1 (all ids) -----------------
     //   d = e_p - rho' e_q   (Z_p (p - q) on the thread's scale),   t = max(d, 0) - c rho' e_q;
     //   S1 += max(-d, 0) = max(d, 0) - d,  S2 += max(-t, 0) = max(t, 0) - t,  R += max(t, 0),  A1 += max(d, 0).
+    // R is also kept per batch: the residual draw then walks one batch of one warp.
     if (needB) {
-        V2 s1 = v2_make(0.f, 0.f), s2 = s1, rr = s1, a1 = s1;
+        V2 s1 = v2_make(0.f, 0.f), s2 = s1, a1 = s1;
+        float Rw = 0.f;
         auto pass_b_batch = [&](int bt, const float (&ep)[32], const float (&eq)[32]) {
             const bool special = hub_warp && (hub_slot >> 2) == bt && hub_slot >= 0;
             const bool any_special = hub_warp && __any_sync(kFull, special);
+            V2 rr = v2_make(0.f, 0.f);
             if (!any_special) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
@@ -754,6 +812,11 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
                     }
                 }
             }
+            if (kSH) {
+                const float rb = warp_sum(mul_ftz(v2_sum(rr), F));
+                push_scalar(&sh.recB[g][4 + bt], rb);
+                Rw += rb;
+            }
         };
 #pragma unroll 1
         for (int bt = 0; bt < LB; ++bt) {
@@ -768,13 +831,20 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             pass_b_batch(LB, ep, eqk);
         }
         const float4 rec[1] = {make_float4(kSH ? warp_sum(mul_ftz(v2_sum(s1), F)) : 0.f,
-                                           kSH ? warp_sum(mul_ftz(v2_sum(s2), F)) : 0.f,
-                                           kSH ? warp_sum(mul_ftz(v2_sum(rr), F)) : 0.f,
+                                           kSH ? warp_sum(mul_ftz(v2_sum(s2), F)) : 0.f, Rw,
                                            kAlg1 ? warp_sum(mul_ftz(v2_sum(a1), F)) : 0.f)};
         res_push<CS, 1>(sh.recB[g], rec, lane);
         res_arrive<CS>();
         res_wait<CS>();   // [2] pass-B records exchanged
     }
+    // The masses of the (warp, batch) parts 8 lane .. 8 lane + 7 of a row, in id order (NB <= 4 per warp).
+    auto parts_of = [&](const float *rec0, int stride, int off, float (&m)[8]) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int gg = 2 * lane + (i >> 2), bt = i & 3;
+            m[i] = (gg < W && bt < NB) ? rec0[gg * stride + off + bt] : 0.f;
+        }
+    };
 
     // ---- warp 0: SpecHub's tests (Algorithm 3); scalars of Algorithm 1's second stage ---------------
     float A1 = 0.f, A1g[3] = {0.f, 0.f, 0.f}, A1grho[3] = {0.f, 0.f, 0.f};
@@ -791,8 +861,9 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
 #pragma unroll
             for (int i = 0; i < 4; ++i) tot[i] = warp_sum(x0[i] + y0[i]);
             if (kSH) {
-                float base = 0.f;
-                selB = res_pick(x0[2], y0[2], ures * tot[2], lane, base);
+                float m[8], base = 0.f;
+                parts_of(&sh.recB[0][0], 8, 4, m);
+                selB = res_pick8(m, ures * tot[2], lane, base);
                 ttB = ures * tot[2] - base;
             }
         }
@@ -839,20 +910,21 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             sh.bc[6] = A1grho[1]; sh.bc[7] = A1grho[2];
         }
     }
-    if (kAlg1 || kSH) __syncthreads();
+    __syncthreads();
 
     // ---- pass C (Algorithm 1): mass of the residual after two rejections ---------------------------
-    //   t = max(d, 0) - A1 q1 / Z...  on the thread's scale:  t = max(d, 0) - (A1 g rho') e_q,  W2 += max(t, 0)
+    //   on the thread's scale:  t = max(d, 0) - (A1 g rho') e_q,  W2 += max(t, 0)
     const float sr_t = kAlg1 ? __fmul_rn(sh.bc[6], sc) : 0.f, sw_t = kAlg1 ? __fmul_rn(sh.bc[7], sc) : 0.f;
     const int x1w_slot = kRW ? cslot[2] : -1;
     const bool x1w_warp = kRW && cwarp[2];
     const int x1w_el = cand[2] & 7;
     if (kAlg1 && needC) {
         const V2 nsr2 = v2_make(-sr_t, -sr_t), nsw2 = v2_make(-sw_t, -sw_t);
-        V2 wr = v2_make(0.f, 0.f), ww = wr;
+        float Wr = 0.f, Ww = 0.f;
         auto pass_c_batch = [&](int bt, const float (&ep)[32], const float (&eq)[32]) {
             const bool special = x1w_warp && x1w_slot >= 0 && (x1w_slot >> 2) == bt;
             const bool any_special = x1w_warp && __any_sync(kFull, special);
+            V2 wr = v2_make(0.f, 0.f), ww = wr;
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
                 const V2 e_q = v2_make(eq[i], eq[i + 1]);
@@ -867,6 +939,16 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
                     ww = v2_add(ww, v2_max0(v2_fma(s, e_q, m)));
                 }
             }
+            if (kR) {
+                const float v = warp_sum(mul_ftz(v2_sum(wr), F));
+                push_scalar(&sh.recC[g][4 + bt], v);
+                Wr += v;
+            }
+            if (kRW) {
+                const float v = warp_sum(mul_ftz(v2_sum(ww), F));
+                push_scalar(&sh.recC[g][8 + bt], v);
+                Ww += v;
+            }
         };
 #pragma unroll 1
         for (int bt = 0; bt < LB; ++bt) {
@@ -880,8 +962,7 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             tmem_ld32(taddr + 32 * LB, ep);
             pass_c_batch(LB, ep, eqk);
         }
-        const float4 rec[1] = {make_float4(kR ? warp_sum(mul_ftz(v2_sum(wr), F)) : 0.f,
-                                           kRW ? warp_sum(mul_ftz(v2_sum(ww), F)) : 0.f, 0.f, 0.f)};
+        const float4 rec[1] = {make_float4(Wr, Ww, 0.f, 0.f)};
         res_push<CS, 1>(sh.recC[g], rec, lane);
         res_arrive<CS>();
         res_wait<CS>();   // [3] pass-C records exchanged
@@ -893,14 +974,13 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             int selC[3] = {-1, -1, -1};
             if (needC) {
                 const int g0 = 2 * lane, g1 = 2 * lane + 1;
-                float x0[2] = {0.f, 0.f}, y0[2] = {0.f, 0.f};
-                if (g0 < W) { x0[0] = sh.recC[g0][0]; x0[1] = sh.recC[g0][1]; }
-                if (g1 < W) { y0[0] = sh.recC[g1][0]; y0[1] = sh.recC[g1][1]; }
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const float tt = warp_sum(x0[i] + y0[i]);
-                    float base = 0.f;
-                    selC[1 + i] = res_pick(x0[i], y0[i], ures * tt, lane, base);
+                    if (!((i == 0 && kR) || (i == 1 && kRW))) continue;
+                    const float tt = warp_sum((g0 < W ? sh.recC[g0][i] : 0.f) + (g1 < W ? sh.recC[g1][i] : 0.f));
+                    float m[8], base = 0.f;
+                    parts_of(&sh.recC[0][0], 12, 4 + 4 * i, m);
+                    selC[1 + i] = res_pick8(m, ures * tt, lane, base);
                     W2raw[1 + i] = tt;
                     ttC[1 + i] = ures * tt - base;
                 }
@@ -943,26 +1023,28 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             if (MASK & (1 << m)) write_node3(A.out[m], r, o[m], elsewhere[m]);
     }
 
-    // ---- residual draws: the warp whose range holds the target walks its stored exponentials ---------
-    // kind: what the weights are.  wsc: -(second-stage scale) on the thread's scale; xex: id whose second-
-    // stage scale is 0 (RRSw's first draft), hubx: id without weight (the hub).
-    auto draw = [&](int kind, int sel, float tt, float nscale, int xex, int hubx, int32_t *token_out) {
-        if (kind == kDrawP) {   // residual mass 0 on a rejection: the token is a draw from p
+    // ---- residual draws: the warp whose range holds the target walks one batch of its stored exponentials
+    // kind: what the weights are.  nscale: -(second-stage scale) on the thread's scale; xex: id whose second-
+    // stage scale is 0 (RRSw's first draft), hubx: id without weight (the hub).  part = 4 * warp + batch.
+    auto draw = [&](int kind, int part, float tt, float nscale, int xex, int hubx, int32_t *token_out) {
+        if (kind == kDrawP) {   // residual mass 0 on a rejection: the token is a draw from p (whole warp ranges)
             if (warp == 0) {
                 const int g0 = 2 * lane, g1 = 2 * lane + 1;
-                const float m0 = g0 < W ? __fmul_rn(sh.recA[g0][1], res_pow2(sh.recA[g0][0] - Cp)) : 0.f;
-                const float m1 = g1 < W ? __fmul_rn(sh.recA[g1][1], res_pow2(sh.recA[g1][0] - Cp)) : 0.f;
-                const float Ztot = warp_sum(m0 + m1);
+                float m[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (g0 < W) m[0] = __fmul_rn(sh.recA[g0][1], res_pow2(sh.recA[g0][0] - Cp));
+                if (g1 < W) m[4] = __fmul_rn(sh.recA[g1][1], res_pow2(sh.recA[g1][0] - Cp));
+                const float Ztot = warp_sum(m[0] + m[4]);
                 float base;
-                const int s = res_pick(m0, m1, ures * Ztot, lane, base);
+                const int s = res_pick8(m, ures * Ztot, lane, base);
                 if (lane == 0) { sh.bi[10] = s; sh.bc[20] = ures * Ztot - base; }
             }
             __syncthreads();
-            sel = sh.bi[10];
+            part = sh.bi[10] < 0 ? -1 : (sh.bi[10] & ~3);   // batch 0 of the picked warp; the walk goes on
             tt = sh.bc[20];
             __syncthreads();
         }
-        if (sel != g) return;
+        if (part < 0 || (part >> 2) != g) return;
+        const int bt0 = part & 3, bt1 = (kind == kDrawP) ? NB : bt0 + 1;
         float prefix = 0.f;
         int found = -1, lastpos = -1;
         const V2 ns2 = v2_make(nscale, nscale);
@@ -993,13 +1075,13 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_verify_kernel(FusedAr
             }
         };
 #pragma unroll 1
-        for (int bt = 0; bt < LB && found < 0; ++bt) {
+        for (int bt = bt0; bt < bt1 && bt < LB && found < 0; ++bt) {
             float ep[32], eq[32];
             tmem_ld32(taddr + 32 * bt, ep);
             load_eq_batch(bt, eq);
             walk(bt, ep, eq);
         }
-        if (found < 0) {
+        if (found < 0 && bt1 > LB) {
             float ep[32];
             tmem_ld32(taddr + 32 * LB, ep);
             walk(LB, ep, eqk);
