@@ -6,6 +6,7 @@ methods, the draft step, the verification of every tree node and the tree walk,
 all on one stream.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
+  python bench.py --workload all      # every configuration and both layouts, one JSON line with a table
 
 Timing: CUDA events on the launching stream, barrier + synchronize on both
 sides, max over ranks.  The headline workloads' inputs (several GB) are far
@@ -34,10 +35,10 @@ METRIC = "tree-nodes verified/sec"
 UNIT = "nodes/s"
 METHODS = ("spechub", "rrs", "rrsw")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per (sequence, node) row, from the ncu capture
-# summarised in profiles/lean_kernels_c4_batch32.md (992 rows); a launch's traffic is this times its
-# row count (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not
-# captured for the current kernels.
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch over 992 (sequence, node) rows of the
+# headline shape, from an ncu capture of the kernels as they stand (the test suite checks these numbers
+# against the committed capture summary); a launch's traffic is this per row times its row count
+# (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not captured.
 TRAFFIC_PER_ROW = {
     ("spechub_draft_sample", "c4"): 275031600.0 / 992,
     ("spechub_verify_tree", "c4"): 941715280.0 / 992,
@@ -54,7 +55,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c4", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--workload", default="c4", choices=sorted(workloads.all_configs()) + ["all"])
     ap.add_argument("--layout", default="dense", choices=["dense", "paper"],
                     help="dense: every node verifies; paper: last-level nodes only draw the bonus token")
     ap.add_argument("--batch", type=int, default=0,
@@ -130,6 +131,34 @@ def oracle_sample(cfg, layout, seconds):
             break
     return done_nodes / spent, "%d whole sequences (%d nodes each) x %d methods, %.1f s" % (
         b, cfg.nodes, len(METHODS), spent), spent
+
+
+def oracle_all_cores(cfg, layout, one_core_rate, seconds):
+    """The same oracle fanned out over the host's cores by ranges of sequences (processes; the oracle
+    itself stays single-threaded).  `one_core_rate` sizes the sample to about `seconds` of wall time."""
+    from oracle import fanout
+
+    n = fanout.cores()
+    per_seq = len(METHODS) * cfg.nodes / max(one_core_rate, 1e-9)          # seconds of one core per sequence
+    S = int(max(n, min(cfg.batch, 4 * n, seconds * n / max(per_seq, 1e-9))))
+    S = min(S, cfg.batch)
+    kind = workloads.paper_node_kind(cfg.nodes) if layout == "paper" else None
+    prior = workloads._prior(cfg)
+    seqs = [workloads.host_sequence(cfg, b, prior) for b in range(S)]
+    lp = np.stack([s[0] for s in seqs]); lq = np.stack([s[1] for s in seqs])
+    un = workloads.host_uniforms(cfg, list(range(S)))
+    del seqs
+    with fanout.Pool(n) as pool:
+        pool.draft_batch("rrs", lq[:n], cfg.temperature, un[:n])             # workers started and warm
+        t0 = time.perf_counter()
+        for m in METHODS:
+            d = pool.draft_batch(m, lq, cfg.temperature, un)
+            pool.verify_batch(m, lp, lq, cfg.temperature, d["tokens"], un, kind)
+        spent = time.perf_counter() - t0
+    return {"value": len(METHODS) * S * cfg.nodes / spent, "unit": UNIT, "cores": n, "kind": "oracle",
+            "sample": "%d whole sequences (%d nodes each) x %d methods over %d worker processes, %.1f s "
+                      "(logits handed over in shared memory, inside the timed region)" % (
+                          S, cfg.nodes, len(METHODS), n, spent)}
 
 
 def run_reference(args, cfg):
@@ -222,9 +251,46 @@ def measured_peak():
     return 6650.0, "fallback (6.65 TB/s)"
 
 
+def run_table(args):
+    """Every configuration (config 3 as its four variants) in both layouts: one bench run each, in a
+    process of its own, gathered into one JSON line.  The headline `value` stays config 4's."""
+    names = ["c1", "c2"] + [v.name for v in workloads.variants("c3")] + ["c4", "c5"]
+    peak, peak_src = measured_peak()
+    table = []
+    for name in names:
+        for layout in ("dense", "paper"):
+            cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--layout", layout,
+                   "--steps", str(args.steps), "--warmup", str(args.warmup), "--e2e-steps", "1",
+                   "--no-cpu-baseline", "--verify-path", args.verify_path]
+            out = subprocess.run(cmd, capture_output=True, text=True)
+            lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+            if out.returncode != 0 or not lines:
+                table.append({"workload": name, "layout": layout, "error": (out.stderr or "no output")[-300:]})
+                continue
+            d = json.loads(lines[-1])
+            k = d["kernels"]
+            table.append({
+                "workload": name, "layout": layout,
+                "nodes_per_s_three_methods": d["value"], "ms_per_step": d["ms_per_step"],
+                "spechub_nodes_per_s": d["breakdown"]["spechub_only_step"]["nodes_per_s"],
+                "spechub_verify_vocab_elements_per_s": d["breakdown"]["spechub_verify_vocab_elements_per_s"],
+                "ms_per_call": {c: k[c]["ms_per_launch"] for c in k},
+                "frac_of_measured_peak": {c: k[c]["frac"] for c in k},
+                "frac_of_8TBs": {c: k[c]["frac_of_nominal_8TBs"] for c in k},
+                "clocks": d.get("clocks"),
+            })
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "table": table, "peak_GBs": peak, "peak_source": peak_src,
+                      "steps": args.steps, "note": "one process per row of the table; fractions are algorithmic "
+                      "bytes / CUDA-event time over the HBM peak"}), flush=True)
+
+
 def main():
     args = parse()
-    cfg = workloads.CONFIGS[args.workload]
+    if args.workload == "all":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_table(args)
+        return
+    cfg = workloads.lookup(args.workload)
     if args.batch:
         from dataclasses import replace as _replace
 
@@ -466,10 +532,14 @@ def main():
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(cfg, args.layout, world),
+            "value_note": "each node is counted once per method (SpecHub, RRS, RRSw run one after another on the "
+                          "same inputs): node-method verifications; SpecHub alone is breakdown.spechub_only_step",
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": args.e2e_steps, "chunks": n_chunks,
                     "note": "pinned host buffers -> device -> public API -> pinned host results; "
-                            "chunks of whole sequences on two streams (copies overlap kernels)"},
+                            "chunks of whole sequences on two streams (copies overlap kernels).  Bound by the "
+                            "host link: the logits (h2d_bytes_per_step) cross it every step, so this is not a "
+                            "kernel number"},
             # per step and method: draft kernel, verification kernel, walk kernel; in paper layout the
             # large-vocabulary bf16 path adds a kernel for the leaf rows
             "gpu_launches": (9 + (3 if args.layout == "paper" and cfg.dtype == "bf16" and cfg.vocab >= 8192
@@ -485,6 +555,12 @@ def main():
                 "peak_ex2_per_s": 148 * 16 * (clocks["sm_mhz"] or 1965.0) * 1e6,
             },
             "breakdown": {
+                "spechub_only_step": {
+                    "ms_per_step": call_ms["spechub_draft_sample"] + call_ms["spechub_verify_tree"],
+                    "nodes_per_s": B * N * world / ((call_ms["spechub_draft_sample"]
+                                                     + call_ms["spechub_verify_tree"]) * 1e-3),
+                    "note": "spechub_draft_sample + spechub_verify_tree (verification and walk kernels) of the "
+                            "timed steps: each node counted once"},
                 "spechub_verify_nodes_per_s": B * N / (verify_ms * 1e-3),
                 "spechub_verify_vocab_elements_per_s": B * N * V / (verify_ms * 1e-3),
                 "step_vocab_elements_per_s": nodes_per_step * V * args.steps / (ms * 1e-3),
@@ -508,6 +584,7 @@ def main():
         if not args.no_cpu_baseline and world == 1:
             v, desc, _ = oracle_sample(cfg, args.layout, args.cpu_seconds)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+            line["cpu_baseline_all_cores"] = oracle_all_cores(cfg, args.layout, v, args.cpu_seconds)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

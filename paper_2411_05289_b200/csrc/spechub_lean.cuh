@@ -94,6 +94,52 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float (&o)[8]) {
     o[6] = __uint_as_float(v.w << 16); o[7] = __uint_as_float(v.w & 0xffff0000u);
 }
 
+// Two fp32 lanes per instruction (fma / add / sub .f32x2): half the issue slots of the scalar forms,
+// the same roundings (round to nearest, subnormals kept), so results do not depend on which form is used.
+struct F2 {
+    unsigned long long v;
+};
+__device__ __forceinline__ F2 f2_make(float lo, float hi) {
+    F2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_get(F2 a, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ F2 f2_fma(F2 a, F2 b, F2 c) {
+    F2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+    return d;
+}
+__device__ __forceinline__ F2 f2_add(F2 a, F2 b) {
+    F2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d.v) : "l"(a.v), "l"(b.v));
+    return d;
+}
+__device__ __forceinline__ F2 f2_sub(F2 a, F2 b) {
+    F2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d.v) : "l"(a.v), "l"(b.v));
+    return d;
+}
+__device__ __forceinline__ F2 f2_max0(F2 a) {
+    float lo, hi;
+    f2_get(a, lo, hi);
+    return f2_make(fmaxf(lo, 0.f), fmaxf(hi, 0.f));
+}
+__device__ __forceinline__ float f2_sum(F2 a) {
+    float lo, hi;
+    f2_get(a, lo, hi);
+    return lo + hi;
+}
+// the exponentials 2^(k l - c) of one 32-bit word (two bf16 logits), as a pair
+__device__ __forceinline__ F2 f2_exp_word(unsigned w, F2 k2, F2 nc2) {
+    const F2 x = f2_fma(f2_make(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)), k2, nc2);
+    float x0, x1;
+    f2_get(x, x0, x1);
+    return f2_make(ex2(x0), ex2(x1));
+}
+
 struct LeanAcc {  // one thread's pass-A state for one row
     unsigned m2;  // packed running maximum
     float c;      // exponent reference (k * some logit of this thread, or 0)
@@ -103,20 +149,19 @@ struct LeanAcc {  // one thread's pass-A state for one row
 __device__ __forceinline__ void lean_push(LeanAcc &st, const uint4 &raw, float k) {
     const unsigned vm = bf2max(bf2max(raw.x, raw.y), bf2max(raw.z, raw.w));
     st.m2 = bf2max(st.m2, vm);
-    float v[8];
-    unpack_bf16x8(raw, v);
-    float e[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) e[i] = ex2(__fmaf_rn(v[i], k, -st.c));
-    float a = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    const F2 k2 = f2_make(k, k);
+    F2 nc2 = f2_make(-st.c, -st.c);
+    // the vector's sum, two lanes at a time: (e0 + e2) + (e4 + e6) and (e1 + e3) + (e5 + e7)
+    float a = f2_sum(f2_add(f2_add(f2_exp_word(raw.x, k2, nc2), f2_exp_word(raw.y, k2, nc2)),
+                            f2_add(f2_exp_word(raw.z, k2, nc2), f2_exp_word(raw.w, k2, nc2))));
     if (!(a < kHuge)) {  // out of range (or NaN / +inf input): move the reference to this vector's max
         const float vmax = bf2_hmax(vm);
         const float cn = shift_of(vmax, k);
         st.s *= ex2(st.c - cn);
         st.c = cn;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) e[i] = ex2(__fmaf_rn(v[i], k, -st.c));
-        a = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+        nc2 = f2_make(-st.c, -st.c);
+        a = f2_sum(f2_add(f2_add(f2_exp_word(raw.x, k2, nc2), f2_exp_word(raw.y, k2, nc2)),
+                          f2_add(f2_exp_word(raw.z, k2, nc2), f2_exp_word(raw.w, k2, nc2))));
     }
     st.s += a;
 }
@@ -894,7 +939,10 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 o.status = 0;  // the full path below sets the flags again
             }
             // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
-            float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
+            // (packed: the low lane takes the even ids of a vector, the high lane the odd ones)
+            F2 s1 = f2_make(0.f, 0.f), s2 = s1, rr = s1;
+            const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ);
+            const F2 nrho2 = f2_make(-rho, -rho), ncrho2 = f2_make(-crho, -crho);
             // software pipeline: the next vector pair is in registers before this one is consumed
             uint4 np = make_uint4(0, 0, 0, 0), nq = np;
             if (last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
@@ -902,23 +950,34 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             for (int vi = last_vi; vi >= lo; vi -= 32) {
                 const uint4 cp = np, cq = nq;
                 if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
-                float fp[8], fq[8];
-                unpack_bf16x8(cp, fp);
-                unpack_bf16x8(cq, fq);
-                if (vi == hubvec) {
+                unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
+                if (vi == hubvec) {   // the hub's own pair is no part of the sums over y != a: -inf, mass 0
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (i == hubel) { fp[i] = neg_inf(); fq[i] = neg_inf(); }
+                    for (int i = 0; i < 4; ++i) {
+                        if (i == (hubel >> 1)) {
+                            const unsigned keep = (hubel & 1) ? 0x0000ffffu : 0xffff0000u;
+                            const unsigned ninf = (hubel & 1) ? 0xff800000u : 0x0000ff80u;
+                            wps[i] = (wps[i] & keep) | ninf;
+                            wqs[i] = (wqs[i] & keep) | ninf;
+                        }
+                    }
                 }
 #pragma unroll
-                for (int i = 0; i < 8; i += 2) {
-                    float d, t;
-                    lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, crho, d, t);
-                    s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
-                    lean_terms(lean_exp(fp[i + 1], k, cP), lean_exp(fq[i + 1], k, cQ), rho, crho, d, t);
-                    s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
+                for (int i = 0; i < 4; ++i) {
+                    const F2 ep = f2_exp_word(wps[i], k2, ncp2), eq = f2_exp_word(wqs[i], k2, ncq2);
+                    const F2 d = f2_fma(nrho2, eq, ep);       // Z_p (p - q)
+                    const F2 m = f2_max0(d);
+                    const F2 t = f2_fma(ncrho2, eq, m);       // Z_p (max(p - q, 0) - c q)
+                    const F2 w = f2_max0(t);
+                    s1 = f2_add(s1, f2_sub(m, d));            // max(-d, 0) = max(d, 0) - d, exactly
+                    s2 = f2_add(s2, f2_sub(w, t));
+                    rr = f2_add(rr, w);
                 }
             }
+            float s1a, s1b, s2a, s2b, ra, rb;
+            f2_get(s1, s1a, s1b);
+            f2_get(s2, s2a, s2b);
+            f2_get(rr, ra, rb);
             float acc[3] = {s1a + s1b, s2a + s2b, ra + rb};
             float part[3][CS];
             lean_row_sums<CS, 3, 0>(acc, part, sh);  // [2]
@@ -984,7 +1043,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
             // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
             const int x1vec = x1 >> 3, x1el = x1 & 7;
-            float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
+            float dna = 0.f, dnb = 0.f;
+            F2 a1 = f2_make(0.f, 0.f);   // (packed: low lane = even ids of a vector, high lane = odd ids)
+            const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ), nrho2 = f2_make(-rho, -rho);
             // RRSw: the next vector pair is loaded before the current one is consumed (measured:
             // 2.21 -> 2.03 ms on V = 128256; for RRS the plain loop unrolled twice is the faster one)
             constexpr bool PIPE = (METHOD == kRRSw);
@@ -999,18 +1060,17 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 } else {
                     cp = vp[vi]; cq = vq[vi];
                 }
-                float fp[8], fq[8];
-                unpack_bf16x8(cp, fp);
-                unpack_bf16x8(cq, fq);
-                float pp[8], qq[8];   // e_p, e_q
+                const unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
+                F2 eq[4];   // e_q of the vector, by words
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
-#pragma unroll
-                for (int i = 0; i < 8; i += 2) {
-                    a1a += fmaxf(__fmaf_rn(-rho, qq[i], pp[i]), 0.f);
-                    a1b += fmaxf(__fmaf_rn(-rho, qq[i + 1], pp[i + 1]), 0.f);
+                for (int i = 0; i < 4; ++i) {
+                    eq[i] = f2_exp_word(wqs[i], k2, ncq2);
+                    a1 = f2_add(a1, f2_max0(f2_fma(nrho2, eq[i], f2_exp_word(wps[i], k2, ncp2))));
                 }
                 if (METHOD == kRRSw) {
+                    float qq[8];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) f2_get(eq[i], qq[2 * i], qq[2 * i + 1]);
                     if (vi == x1vec) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
@@ -1020,6 +1080,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     dnb += (qq[4] + qq[5]) + (qq[6] + qq[7]);
                 }
             }
+            float a1a, a1b;
+            f2_get(a1, a1a, a1b);
             float acc[2] = {a1a + a1b, dna + dnb};
             float part2[2][CS];
             lean_row_sums<CS, 2, 0>(acc, part2, sh);  // [2]
@@ -1029,7 +1091,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             const float A1g = A1 * gq;
             const float A1grho = A1g * rho;
             // pass C: mass of the residual after two rejections
-            float w2a = 0.f, w2b = 0.f;
+            F2 w2 = f2_make(0.f, 0.f);
+            const F2 nsc2 = f2_make(-A1grho, -A1grho);
             if (PIPE && lo + lane < hi) { np = vp[lo + lane]; nq = vq[lo + lane]; }
 #pragma unroll(PIPE ? 1 : 2)
             for (int vi = lo + lane; vi < hi; vi += 32) {
@@ -1040,30 +1103,23 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 } else {
                     cp = vp[vi]; cq = vq[vi];
                 }
-                float fp[8], fq[8];
-                unpack_bf16x8(cp, fp);
-                unpack_bf16x8(cq, fq);
-                float sc[8];
+                const unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
+                const bool x1here = (METHOD == kRRSw && vi == x1vec);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sc[i] = A1grho;
-                if (METHOD == kRRSw && vi == x1vec) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (i == x1el) sc[i] = 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < 8; i += 2) {
-                    float d, t;
-                    lean_terms(lean_exp(fp[i], k, cP), lean_exp(fq[i], k, cQ), rho, sc[i], d, t);
-                    w2a += fmaxf(t, 0.f);
-                    lean_terms(lean_exp(fp[i + 1], k, cP), lean_exp(fq[i + 1], k, cQ), rho, sc[i + 1], d, t);
-                    w2b += fmaxf(t, 0.f);
+                for (int i = 0; i < 4; ++i) {
+                    F2 nsc = nsc2;
+                    if (x1here && i == (x1el >> 1)) nsc = (x1el & 1) ? f2_make(-A1grho, 0.f) : f2_make(0.f, -A1grho);
+                    const F2 eq = f2_exp_word(wqs[i], k2, ncq2);
+                    const F2 m = f2_max0(f2_fma(nrho2, eq, f2_exp_word(wps[i], k2, ncp2)));
+                    w2 = f2_add(w2, f2_max0(f2_fma(nsc, eq, m)));
                 }
             }
-            float w2[1] = {w2a + w2b};
+            float w2a, w2b;
+            f2_get(w2, w2a, w2b);
+            float w2s[1] = {w2a + w2b};
             float part1[1][CS];
-            lean_row_sums<CS, 1, 2>(w2, part1, sh);  // [3]
-            const float W2raw = w2[0], W2 = W2raw * invZp;
+            lean_row_sums<CS, 1, 2>(w2s, part1, sh);  // [3]
+            const float W2raw = w2s[0], W2 = W2raw * invZp;
             o.rate[0] = fmaxf(1.f - A1, 0.f);
             o.rate[1] = fmaxf(A1 - W2, 0.f);
             o.rate[2] = W2;

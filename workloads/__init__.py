@@ -72,6 +72,18 @@ def variants(name: str):
     return out
 
 
+def all_configs():
+    """Every configuration by name, config 3's four variants included (and its base, c3)."""
+    out = dict(CONFIGS)
+    for v in variants("c3"):
+        out[v.name] = v
+    return out
+
+
+def lookup(name: str) -> Config:
+    return all_configs()[name]
+
+
 # ---- bf16 <-> fp32 on the host (numpy has no bf16) ------------------------------------------------
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
