@@ -60,9 +60,10 @@ def parse():
                     help="dense: every node verifies; paper: last-level nodes only draw the bonus token")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch (profiling on a small case; not a bench value)")
-    ap.add_argument("--verify-path", default="default", choices=["default", "streaming", "resident"],
+    ap.add_argument("--verify-path", default="default", choices=["default", "streaming", "split2", "split4", "resident"],
                     help="large-vocabulary verification kernels: the library's choice, the two-pass streaming "
-                         "kernels, or the kernels that keep the exponentials on chip")
+                         "kernels (one CTA per row, or a row split over 2 / 4 CTAs), or the kernels that keep the "
+                         "exponentials on chip")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle timing leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -314,7 +315,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     sh.load_library()
-    sh.set_row_split({"default": 0, "streaming": 1, "resident": 8}[args.verify_path])
+    sh.set_row_split({"default": 0, "streaming": 1, "split2": 2, "split4": 4, "resident": 8}[args.verify_path])
 
     # this rank's batch (same shape on every rank, its own seed)
     from dataclasses import replace

@@ -577,3 +577,30 @@ def test_unbalanced_tree_from_parents(sh):
             for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
                 np.testing.assert_array_equal(out[k], w[k], err_msg="unbalanced walk %s" % k)
             assert out["n_accepted"].max() >= 2
+
+
+def test_walk_stops_at_an_accept_index_outside_the_children(sh):
+    """spechub_walk_tree takes a caller-supplied accept_idx (the vocabulary-sharded path hands it the
+    exchanged array): an index that names no child ends the walk at that node instead of indexing
+    past the child table."""
+    import ctypes
+
+    from paper_2411_05289_b200 import binding, vocab_sharded
+
+    lib = vocab_sharded._lib()
+    B, N = 3, 7
+    tree = sh.Tree.heap(N)
+    x = torch.zeros((B, N, 64), dtype=torch.float32, device="cuda")
+    d, _ = binding._desc(x, tree, 1.0)
+    acc = torch.tensor([[0, 2, 0, 0, 0, 0, 0], [1, 0, 2147483647, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0, 0]],
+                       dtype=torch.int32, device="cuda")
+    tok = torch.arange(B * N, dtype=torch.int32, device="cuda").reshape(B, N) + 100
+    out = binding.alloc_verify_outputs(B, N, tree.levels, x.device)
+    so = binding._SeqOut(*[out[k].data_ptr() for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens")])
+    rc = lib.spechub_walk_tree(ctypes.byref(d), ctypes.c_void_p(acc.data_ptr()), ctypes.c_void_p(tok.data_ptr()),
+                               ctypes.byref(so), None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert out["path_nodes"].cpu().tolist() == [[0, 1, -1], [0, 2, -1], [0, 1, 4]]
+    assert out["n_accepted"].cpu().tolist() == [1, 1, 3]
+    assert out["n_emitted"].cpu().tolist() == [2, 2, 3]
