@@ -10,11 +10,15 @@ Probabilities: |gpu - oracle| <= RTOL * |oracle| + floor, RTOL = 1e-5, with a
 floor of 1e-12 for values below 1e-7.  Two kinds of output are not plain sums
 of positive terms and carry a further, derived, term:
 
-  * rate[0] and rate[1] are differences of O(1) sums (e.g. the mass accepted at
-    child 0 is (1 - q(a)) - S1 + min(p(a), S2)): each sum carries a few fp32
-    ulps times log2(V) of summation error, about 1e-6 absolute on quantities
-    bounded by 1.  They get ATOL_DIFF = 1e-6.  rate[2] (a sum of non-negative
-    terms) gets none.
+  * the rates are built from differences of probabilities: rate[0] and rate[1]
+    are differences of O(1) sums (e.g. the mass accepted at child 0 is
+    (1 - q(a)) - S1 + min(p(a), S2)), and every term of rate[2] is a clipped
+    difference max(p - q - c q, 0) whose operands (p, q, c q: each family sums
+    to at most 1) carry the fp32 error of a single probability.  So a rate has
+    an absolute error of a few 1e-7 whatever its size, and a small rate cannot
+    meet a relative bar (a rejection mass of 2e-4 on a two-token vocabulary was
+    off by 1e-8: 5e-5 relative).  They get ATOL_DIFF = 1e-6; the measurement
+    below records how little of it is used.
   * an acceptance probability N/D whose numerator is a difference (p(x) - q(x),
     p(a) - S2) is ill-conditioned when the operands nearly cancel: a relative
     error EPS in every fp32 p(y), q(y) moves N/D by EPS * cond, where cond is
@@ -40,7 +44,7 @@ import oracle
 NEAR = 1e-6
 RTOL = 1e-5
 FLOOR = 1e-12       # absolute floor, for values below 1e-7
-ATOL_DIFF = 1e-6    # rate[0], rate[1]: differences of O(1) sums
+ATOL_DIFF = 1e-6    # the rates: sums of (clipped) differences of probabilities
 ATOL = ATOL_DIFF    # (the k-draft rates m_j - m_{j+1} are differences too)
 EPS = 1e-6
 
@@ -191,7 +195,7 @@ def check_verify_row(method, lp_row, lq_row, T, tokens, u, leaf, g, o, ctx, stat
         _close(g["beta"][i], o["beta"][i], "beta[%d]" % i, ctx, stats, extra=EPS * float(o["cond"][i]))
     _close(g["rate"][0], o["rate"][0], "rate[0]", ctx, stats, extra=ATOL_DIFF)
     _close(g["rate"][1], o["rate"][1], "rate[1]", ctx, stats, extra=ATOL_DIFF)
-    _close(g["rate"][2], o["rate"][2], "rate[2]", ctx, stats)
+    _close(g["rate"][2], o["rate"][2], "rate[2]", ctx, stats, extra=ATOL_DIFF)
     if g["accept_idx"] == o["accept_idx"] and g["token"] == o["token"]:
         stats.exact += 1
         soft = oracle.STATUS_BITS["ZERO_RESIDUAL"]
