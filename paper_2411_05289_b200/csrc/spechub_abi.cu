@@ -13,6 +13,7 @@
 #include "spechub_kary.cuh"
 #include "spechub_fused.cuh"
 #include "spechub_resident.cuh"
+#include "spechub_resident_kary.cuh"
 #include "spechub_shard.cuh"
 #include "spechub_shard_rrs.cuh"
 
@@ -142,9 +143,15 @@ bool lean_ok(const spechub_desc *d, bool aligned) {
 // cluster that holds the row with at most four batches per lane is taken.
 struct ResShape { int cs, nb; };
 
+bool resident_fits(const spechub_desc *d, bool aligned, ResShape *out);
+
+// two drafts per node: on request (SPECHUB_FLAG_RESIDENT)
 bool resident_shape(const spechub_desc *d, bool aligned, ResShape *out) {
+    return (d->flags & SPECHUB_FLAG_RESIDENT) && resident_fits(d, aligned, out);
+}
+
+bool resident_fits(const spechub_desc *d, bool aligned, ResShape *out) {
     if (!lean_ok(d, aligned)) return false;
-    if (!(d->flags & SPECHUB_FLAG_RESIDENT)) return false;
     const int nvec = d->vocab / 8;
     for (int cs = 1; cs <= 8; cs *= 2) {
         const int parts = cs * kResWarps;
@@ -196,6 +203,43 @@ int launch_resident_mask(ResShape sh, const FusedArgs &f, unsigned rows, cudaStr
     if (sh.cs == 2) return launch_resident_one<MASK, 2>(sh.nb, f, rows, s);
     if (sh.cs == 4) return launch_resident_one<MASK, 4>(sh.nb, f, rows, s);
     return launch_resident_one<MASK, 8>(sh.nb, f, rows, s);
+}
+
+// Algorithm 1 with k > 2 drafts: the stages run over the exponentials kept on chip
+template <int CS>
+int launch_resident_kary_one(int nb, const KaryArgs &ka, unsigned rows, cudaStream_t s) {
+    auto kern = resident_kary_kernel<CS>;
+    const uint32_t cols = nb == 1 ? 64u : nb == 2 ? 128u : 256u;
+    int smem = (nb - 1) * 4 * 2 * kResThreads * 16;
+    if (cols == 256u && smem < 76 * 1024) smem = 76 * 1024;   // at most two CTAs of 256 columns per SM
+    constexpr int smem_max = (kResMaxBatches - 1) * 4 * 2 * kResThreads * 16;
+    static bool configured[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECHUB_ERR_LAUNCH;
+    {
+        std::lock_guard<std::mutex> lock(g_attr_mutex);
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) {
+                cudaGetLastError();
+                return SPECHUB_ERR_LAUNCH;
+            }
+            configured[dev] = true;
+        }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = CS > 1 ? 1 : 0;
+    cfg.gridDim = dim3(rows * CS); cfg.blockDim = dim3(kResThreads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    return cudaLaunchKernelEx(&cfg, kern, ka, nb, cols) == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+}
+
+int launch_resident_kary(ResShape sh, const KaryArgs &ka, unsigned rows, cudaStream_t s) {
+    if (sh.cs == 1) return launch_resident_kary_one<1>(sh.nb, ka, rows, s);
+    if (sh.cs == 2) return launch_resident_kary_one<2>(sh.nb, ka, rows, s);
+    if (sh.cs == 4) return launch_resident_kary_one<4>(sh.nb, ka, rows, s);
+    return launch_resident_kary_one<8>(sh.nb, ka, rows, s);
 }
 
 // mask: bit m set = method m (0 SpecHub, 1 RRS, 2 RRSw) is verified; leaf rows go to lean_leaf_kernel
@@ -325,7 +369,11 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
         if (method == kSpecHub) return SPECHUB_ERR_SHAPE;
         KaryArgs ka;
         ka.r = a; ka.k = d->k; ka.without_replacement = (method == kRRSw);
-        if (d->dtype == SPECHUB_BF16) {
+        ResShape rs;
+        if (!(d->flags & 7u) && resident_fits(d, al, &rs)) {   // (a split flag asks for the streaming kernel)
+            const int lrc = launch_resident_kary(rs, ka, rows, s);
+            if (lrc != SPECHUB_OK) return lrc;
+        } else if (d->dtype == SPECHUB_BF16) {
             if (al) kary_verify_kernel<__nv_bfloat16, true><<<rows, th, 0, s>>>(ka);
             else kary_verify_kernel<__nv_bfloat16, false><<<rows, th, 0, s>>>(ka);
         } else {
