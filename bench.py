@@ -64,6 +64,9 @@ def parse():
                     help="large-vocabulary verification kernels: the library's choice, the two-pass streaming "
                          "kernels (one CTA per row, or a row split over 2 / 4 CTAs), or the kernels that keep the "
                          "exponentials on chip")
+    ap.add_argument("--kary-leg", action="store_true",
+                    help="also time RRS / RRSw with three drafts per node on a ternary 40-node tree of the "
+                         "workload's vocabulary (reported in breakdown, not part of `value`)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle timing leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -84,6 +87,10 @@ def config_dict(cfg, layout, n_gpus):
 
 
 L2_BYTES = 126e6
+
+
+def esz0(cfg):
+    return 2 if cfg.dtype == "bf16" else 4
 
 
 def input_bytes(cfg):
@@ -449,6 +456,34 @@ def main():
     else:
         graph_note = "same nine launches per step, replayed from %d captured graph(s); not part of `value`" % len(copies)
 
+    # ---- extra: Algorithm 1 with three drafts per node (the paper's ternary trees) ----
+    kary = None
+    if args.kary_leg:
+        t3 = sh.Tree.kary(3, 4, device=dev)
+        N3 = t3.nodes_of_complete_tree()
+        gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 3)
+        dt = tp.dtype
+        kp = (torch.randn((B, N3, V), device=dev, generator=gen) * 2.0).to(dt)
+        kq = (kp.float() + torch.randn((B, N3, V), device=dev, generator=gen)).to(dt)
+        ku = (torch.randint(0, 1 << 24, (B, N3, 7), device=dev, generator=gen).float() * 2.0 ** -24)
+        kary = {"tree": "ternary, 4 levels, %d nodes" % N3, "batch": B, "vocab": V,
+                "alg_bytes_per_verify": B * N3 * (2 * V * esz0(cfg) + 12 + 28 + 44)}
+        for wo in (False, True):
+            kd = sh.rrs_draft_sample(kq, ku, t3, wo, cfg.temperature)
+            ko = alloc_verify_outputs(B, N3, t3.levels, dev, 3)
+            for _ in range(3):
+                sh.rrs_verify_tree(kp, kq, kd["tokens"], ku, t3, wo, cfg.temperature, out=ko)
+            barrier()
+            q0.record(stream)
+            for _ in range(args.steps):
+                sh.rrs_verify_tree(kp, kq, kd["tokens"], ku, t3, wo, cfg.temperature, out=ko)
+            q1.record(stream)
+            barrier()
+            t_ms = q0.elapsed_time(q1) / args.steps
+            kary["rrsw" if wo else "rrs"] = {"verify_ms": t_ms, "nodes_per_s": B * N3 / (t_ms * 1e-3),
+                                             "algorithmic_GBs": kary["alg_bytes_per_verify"] / (t_ms * 1e-3) / 1e9}
+        del kp, kq, ku
+
     # ---- end to end: host buffers in, host results out, through the public API ----
     esz = 2 if cfg.dtype == "bf16" else 4
     h_tp = torch.empty(tp.shape, dtype=tp.dtype, pin_memory=True); h_tp.copy_(tp)
@@ -573,6 +608,7 @@ def main():
                     "ms_per_step": graph_ms,
                     "nodes_per_s": (len(METHODS) * B * N / (graph_ms * 1e-3)) if graph_ms else None,
                     "note": graph_note},
+                "three_drafts_per_node": kary,
                 "step_through_three_method_calls": {
                     "ms_per_step": fused_ms, "nodes_per_s": len(METHODS) * B * N / (fused_ms * 1e-3),
                     "gpu_launches_per_step": 5,

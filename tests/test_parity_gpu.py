@@ -455,7 +455,7 @@ def test_config3_sampled(sh, pool, variant):
     report(cfg.name, s)
 
 
-@pytest.mark.parametrize("split,n_sample", [(0, 1024), (4, 128)])
+@pytest.mark.parametrize("split,n_sample", [(0, 4096), (8, 512), (4, 128)])
 def test_config4_sampled(sh, pool, split, n_sample):
     """The default path on 1024+ rows per method and layout; the forced-split streaming kernels on fewer."""
     cfg = workloads.CONFIGS["c4"]
@@ -480,7 +480,7 @@ def test_config5_sampled(sh, pool):
                 per_kind[k].append(b * cfg.nodes + n)
     assert len(per_kind) == len(workloads.ADV_KINDS)
     extra = [(r, k) for k, rows in per_kind.items() for r in rows]
-    s = sampled_parity(sh, cfg, 1024, extra_rows=[e[0] for e in extra], pool=pool)
+    s = sampled_parity(sh, cfg, 2048, extra_rows=[e[0] for e in extra], pool=pool)
     report("c5", s)
 
 
