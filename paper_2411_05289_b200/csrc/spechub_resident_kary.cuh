@@ -68,12 +68,30 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_kary_kernel(KaryArgs 
         lpx[i] = load_one<__nv_bfloat16>(rowp, ok ? x[i] : 0);
         lqx[i] = load_one<__nv_bfloat16>(rowq, ok ? x[i] : 0);
     }
-    // does this warp's range hold one of the drafts (RRSw zeroes them stage by stage)?
-    bool tok_warp = false;
+    // RRSw takes the drafts out of q stage by stage.  Where a draft lies in what this lane stores:
+    // one bit per stored exponential of a batch (bit = 8 * vector of the batch + element).
+    bool tok_warp = false;           // this warp's range holds one of x_1..x_{k-1}
+    auto tok_bit = [&](int i, int &bt) -> unsigned {   // draft i in this lane's storage: its batch and bit, or 0
+        const int v = x[i] >> 3;
+        if (!(x[i] >= 0 && v >= lo && v < hi && ((v - lo) & 31) == lane)) return 0u;
+        const int slot = (v - lo) >> 5;
+        bt = slot >> 2;
+        return 1u << ((slot & 3) * 8 + (x[i] & 7));
+    };
+    auto mask_of = [&](const unsigned (&mk)[4], int bt) {
+        return bt == 0 ? mk[0] : bt == 1 ? mk[1] : bt == 2 ? mk[2] : mk[3];
+    };
+    unsigned mask_all[4] = {0u, 0u, 0u, 0u};   // x_1..x_{k-1}: left out of the sum that gives the renormalisers
+    unsigned mask_cum[4] = {0u, 0u, 0u, 0u};   // the drafts drawn before the current stage
     if (wo && !leaf) {
-        for (int i = 0; i < K; ++i) {
+        for (int i = 0; i < K - 1; ++i) {
             const int v = x[i] >> 3;
             tok_warp |= (x[i] >= 0 && v >= lo && v < hi);
+            int bt = 0;
+            const unsigned bit = tok_bit(i, bt);
+#pragma unroll
+            for (int b4 = 0; b4 < 4; ++b4)
+                if (b4 == bt) mask_all[b4] |= bit;
         }
     }
 
@@ -187,11 +205,9 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_kary_kernel(KaryArgs 
 #pragma unroll
                     for (int i = 0; i < 32; ++i) e[i] = eqk[i];
                 }
+                const unsigned mk = mask_of(mask_all, bt);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int id = (lo + lane + 32 * (4 * bt + (i >> 3))) * 8 + (i & 7);
-                    s0 += in_set(x, K - 1, id) ? 0.f : e[i];
-                }
+                for (int i = 0; i < 32; ++i) s0 += ((mk >> i) & 1u) ? 0.f : e[i];
             }
             sxw = warp_sum(__fmul_rn(s0, fqw));
         }
@@ -273,6 +289,13 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_kary_kernel(KaryArgs 
             const V2 nc2 = v2_make(-ct, -ct);
             float Mw = 0.f;
             float *recs = sh.recS[j & 1][g];
+            if (tok_warp && j > 1) {   // x_{j-1} leaves q from this stage on
+                int btk = 0;
+                const unsigned bit = tok_bit(j - 2, btk);
+#pragma unroll
+                for (int b4 = 0; b4 < 4; ++b4)
+                    if (b4 == btk) mask_cum[b4] |= bit;
+            }
             for (int bt = 0; bt < NB; ++bt) {
                 float P[32], eq[32];
                 tmem_ld32(taddr + 32 * bt, P);
@@ -284,11 +307,10 @@ __global__ void __launch_bounds__(kResThreads, 2) resident_kary_kernel(KaryArgs 
                 }
                 V2 acc = v2_make(0.f, 0.f);
                 if (tok_warp && j > 1) {   // RRSw: drafts drawn before this stage carry no draft mass in it
+                    const unsigned mk = mask_of(mask_cum, bt);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int id = (lo + lane + 32 * (4 * bt + (i >> 3))) * 8 + (i & 7);
-                        if (in_set(x, j - 1, id)) eq[i] = 0.f;
-                    }
+                    for (int i = 0; i < 32; ++i)
+                        if ((mk >> i) & 1u) eq[i] = 0.f;
                 }
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
