@@ -40,12 +40,12 @@ METHODS = ("spechub", "rrs", "rrsw")
 # against the committed capture summary); a launch's traffic is this per row times its row count
 # (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not captured.
 TRAFFIC_PER_ROW = {
-    ("spechub_draft_sample", "c4"): 275031600.0 / 992,
-    ("spechub_verify_tree", "c4"): 941715280.0 / 992,
-    ("rrs_draft_sample[rrs]", "c4"): 278423376.0 / 992,
-    ("rrs_verify_tree[rrs]", "c4"): 1319892128.0 / 992,
-    ("rrs_draft_sample[rrsw]", "c4"): 279134568.0 / 992,
-    ("rrs_verify_tree[rrsw]", "c4"): 1330579352.0 / 992,
+    ("spechub_draft_sample", "c4"): 275403008.0 / 992,
+    ("spechub_verify_tree", "c4"): 939372696.0 / 992,
+    ("rrs_draft_sample[rrs]", "c4"): 278545920.0 / 992,
+    ("rrs_verify_tree[rrs]", "c4"): 1323653824.0 / 992,
+    ("rrs_draft_sample[rrsw]", "c4"): 279179008.0 / 992,
+    ("rrs_verify_tree[rrsw]", "c4"): 1332738336.0 / 992,
 }
 
 
@@ -560,7 +560,8 @@ def main():
             roof[name] = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
                           "frac": ach / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0,
                           "traffic": (TRAFFIC_PER_ROW[(name, args.workload)] * B * N
-                                      if (name, args.workload) in TRAFFIC_PER_ROW and args.layout == "dense" else None),
+                                      if (name, args.workload) in TRAFFIC_PER_ROW and args.layout == "dense"
+                                      and args.verify_path == "default" else None),
                           "alg_bytes_per_launch": nbytes,
                           "ms_per_launch": t_ms, "share_of_step": t_ms / total_call_ms}
         line = {

@@ -42,3 +42,23 @@ def test_gpu_arm_has_no_cpu_fallback():
     r = run("--workload", "c1", "--steps", "1", env={"CUDA_VISIBLE_DEVICES": ""})
     assert r.returncode != 0
     assert "CUDA" in (r.stderr + r.stdout)
+
+
+def test_measured_traffic_matches_the_committed_capture():
+    """bench.py's DRAM traffic per row is typed in from an ncu capture: the numbers must be the ones in the
+    capture's summary, whose header names the commit of the kernels it was taken on."""
+    import importlib.util
+
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    text = open(os.path.join(ROOT, "profiles", "lean_kernels_c4_batch32.md")).read()
+    assert "Kernel sources as of commit" in text
+    row = [l for l in text.splitlines() if l.startswith("| DRAM bytes read + written per launch")]
+    assert len(row) == 1
+    vals = [float(v) for v in row[0].split("|")[2:-1]]
+    calls = ["spechub_draft_sample", "rrs_draft_sample[rrs]", "rrs_draft_sample[rrsw]",
+             "spechub_verify_tree", "rrs_verify_tree[rrs]", "rrs_verify_tree[rrsw]"]
+    assert len(vals) == len(calls)
+    for c, v in zip(calls, vals):
+        assert bench.TRAFFIC_PER_ROW[(c, "c4")] == pytest.approx(v / 992, rel=1e-9), c

@@ -39,10 +39,11 @@ def pool():
         yield p
 
 
-# Rows a full-size configuration may leave to the near-threshold rule: a uniform falls within 1e-6 of
-# one of ~10^5 CDF edges of a row about one time in ten, so a few per cent of rows are expected there;
-# a fraction far above that means the rule is hiding something.
-MAX_EXEMPT_FRACTION = 0.15
+# Rows a full-size configuration may leave to the near-threshold rule.  Measured on configs 1-5: at
+# most 0.43 % of the rows, all of them residual or draft draws whose uniform lies within 1e-6 of an
+# edge of the oracle's CDF (tens of thousands of edges per row); no acceptance test was exempted.  A
+# fraction far above that means the rule is hiding something.
+MAX_EXEMPT_FRACTION = 0.02
 
 
 def report(name, s):
