@@ -538,10 +538,39 @@ def main():
     barrier()
     e2e_s = g0.elapsed_time(g1) * 1e-3
 
-    tms = torch.tensor([ms, e2e_s * 1e3, verify_ms], device=dev, dtype=torch.float64)
+    # ---- several GPUs only: the same SpecHub step with the VOCABULARY sharded over the ranks (a tensor-
+    # parallel LM head): every rank holds an id range of the same rows, runs the phase kernels on its own
+    # slice and exchanges 32 bytes per row between them (two all-gathers and one maximum per call over
+    # NCCL; no kernel is given a peer's memory).  Reported beside the batch-sharded headline.
+    vs_ms = None
+    if world > 1:
+        from paper_2411_05289_b200 import vocab_sharded as vsh
+
+        ctp, ctq = workloads.device_logits(cfg, device=dev)      # the common rows: same seed on every rank
+        cun = workloads.device_uniforms(cfg, device=dev)
+        shard, sp = vsh.slice_of_rank(ctp, rank, world)
+        _, sq = vsh.slice_of_rank(ctq, rank, world)
+        del ctp, ctq
+
+        def vs_step():
+            d = vsh.spechub_draft_sample_sharded(sq, cun, tree, shard, cfg.temperature)
+            return vsh.spechub_verify_tree_sharded(sp, sq, d["tokens"], cun, tree, shard, cfg.temperature)
+
+        for _ in range(3):
+            vs_step()
+        barrier()
+        q0.record(stream)
+        for _ in range(args.steps):
+            vs_step()
+        q1.record(stream)
+        barrier()
+        vs_ms = q0.elapsed_time(q1) / args.steps
+        del sp, sq
+
+    tms = torch.tensor([ms, e2e_s * 1e3, verify_ms, vs_ms or 0.0], device=dev, dtype=torch.float64)
     if world > 1:
         dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, verify_ms = [float(x) for x in tms.tolist()]
+    ms, e2e_ms, verify_ms, vs_ms = [float(x) for x in tms.tolist()]
 
     if rank == 0:
         nodes_per_step = len(METHODS) * B * N * world
@@ -610,6 +639,11 @@ def main():
                     "nodes_per_s": (len(METHODS) * B * N / (graph_ms * 1e-3)) if graph_ms else None,
                     "note": graph_note},
                 "three_drafts_per_node": kary,
+                "vocab_sharded_step": None if world == 1 else {
+                    "ms_per_step": vs_ms, "nodes_per_s": B * N / (vs_ms * 1e-3), "ranks": world,
+                    "nccl_version": ".".join(str(v) for v in torch.cuda.nccl.version()),
+                    "note": "SpecHub draft + verify + walk of ONE batch of %d sequences whose vocabulary is sharded "
+                            "over the ranks (strong scaling of one step); max over ranks; not part of `value`" % B},
                 "step_through_three_method_calls": {
                     "ms_per_step": fused_ms, "nodes_per_s": len(METHODS) * B * N / (fused_ms * 1e-3),
                     "gpu_launches_per_step": 5,

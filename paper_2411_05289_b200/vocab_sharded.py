@@ -280,6 +280,16 @@ def shard_of_group(width: int, group=None) -> Shard:
     return Shard(r, n, sum(widths[:r]), sum(widths))
 
 
+def slice_of_rank(logits, rank: int, nranks: int):
+    """This rank's share of full-vocabulary logits [B][N][V] (a tensor-parallel LM head would hand
+    every rank exactly this): the Shard of ``even_shards`` and a contiguous copy of its id range, so
+    that each rank's kernels read its own memory only.  Slices are 16-byte aligned when the width is
+    a multiple of 8 bf16 ids."""
+    V = logits.shape[-1]
+    shard, width = even_shards(V, nranks)[rank]
+    return shard, logits[..., shard.id_offset:shard.id_offset + width].contiguous()
+
+
 def _on(stream):
     """The drivers below mix kernel launches, allocations and collectives; all of them follow torch's
     current stream, so a caller's stream is made current for the whole call (kernels launched on one

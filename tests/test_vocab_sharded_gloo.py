@@ -65,6 +65,48 @@ def test_exchanges_world_size_2():
     assert (m0[0, :, 0] == 100).all() and (m0[1, :, 0] == 101).all() and (m0[..., 1] == -2).all()
 
 
+def _slice_worker(rank, world, port, q):
+    import torch.distributed as dist
+
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # every rank builds the same full rows (the benchmark's vocabulary-sharded leg does so from a
+        # common seed) and keeps its own id range
+        g = torch.Generator().manual_seed(5)
+        full = torch.randn((2, 3, 1001), generator=g)
+        shard, mine = vs.slice_of_rank(full, rank, world)
+        assert mine.is_contiguous() and mine.shape == (2, 3, 501 if rank == 0 else 500)
+        assert vs.shard_of_group(mine.shape[-1]) == shard          # the ranks agree on the bookkeeping
+        # the slices, gathered in rank order, are the full rows again (pad to a common width to gather)
+        pad = torch.zeros((2, 3, 501))
+        pad[..., : mine.shape[-1]] = mine
+        parts = vs.all_gather_ranks(pad)
+        back = torch.cat([parts[0], parts[1][..., :500]], dim=-1)
+        q.put((rank, bool(torch.equal(back, full))))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_vocabulary_slices_of_the_bench_leg_world_size_2():
+    import torch.multiprocessing as mp
+
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_slice_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted([q.get(timeout=120) for _ in procs])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == [(0, True), (1, True)]
+
+
 def test_even_shards_cover_the_vocabulary():
     from paper_2411_05289_b200 import vocab_sharded as vs
 
