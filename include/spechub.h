@@ -25,7 +25,8 @@
  *     at any data pointer.
  *   - Per-row problems found on the device are reported as bits in the row's
  *     `status` word and give the documented fallback output; kernels never
- *     trap and wait only on hardware barriers.
+ *     trap and wait only on hardware barriers (and, where stated, on the
+ *     hardware's tensor-memory allocator).
  *   - Layout: logits are [batch][nodes][vocab] with element strides
  *     `stride_seq`, `stride_node` (rows are contiguous in the vocabulary).
  *     Rows that start on a 16-byte boundary are read with 128-bit loads; other
@@ -92,7 +93,11 @@ extern "C" {
 #define SPECHUB_FLAG_SPLIT_4 4u
 /* Verification with the exponentials resident on chip (tensor memory + shared memory): one read of the
  * row pair from HBM instead of two.  Not combined with a split flag.  Applies to the same shapes as the
- * large-vocabulary bf16 kernels, up to 262144 ids; other shapes ignore it. */
+ * large-vocabulary bf16 kernels, up to 262144 ids; other shapes ignore it.  These kernels allocate
+ * tensor memory (tcgen05.alloc) for the lifetime of a CTA and release it before the CTA ends; among
+ * themselves they never ask an SM for more than it has.  Another kernel that holds tensor memory on
+ * the same SMs at the same time (a tensor-core GEMM on another stream) makes their CTAs wait until its
+ * CTAs have finished -- a delay, not a deadlock. */
 #define SPECHUB_FLAG_RESIDENT 8u
 
 /* node kinds */
@@ -217,6 +222,10 @@ int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
  * q_j = q (RRS) or q with q(x_1..x_{j-1}) zeroed and renormalised (RRSw),
  * P_j = max(P_{j-1} - m_{j-1} q_j, 0) and m_j = sum P_j; the residual token is
  * drawn from P_k; rate[j] = m_j - m_{j+1} (j < k), rate[k] = m_k.
+ * For desc->k > 2 on bf16 rows that are 16-byte aligned with 8192 <= vocab <=
+ * 262144, vocab % 8 == 0 and no split flag, the stages run over exponentials
+ * kept in the SMs' tensor memory and shared memory (see SPECHUB_FLAG_RESIDENT
+ * for what that means for other work on the GPU).
  */
 int rrs_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
                     const int32_t *draft_tokens, const float *uniforms, int without_replacement,

@@ -11,7 +11,10 @@ captions of Figures 4 and 5, exactness of the emitted token's law (Theorem 2)
 by enumeration for V <= 8, the closed form against a brute-force LP on
 SpecHub's support (Section 3.2), hub mass = p(a) (Corollary 1), Theorem 3's
 ordering against RRS, the T -> 0 top-2 limit (Section 5.2), and the
-degenerate rows.  Nothing in this package is "parity unpinned".
+degenerate rows; ``cond`` (the conditioning figure the parity checker sizes its tolerance with)
+against the derivatives of the oracle's own acceptance ratios (``tests/test_oracle_cond.py``).
+``fanout`` runs the batch calls on several cores (same results, bit for bit).  Parity unpinned: the
+printed digits of the paper's toy table only (``toy_table.py``).
 """
 from .oracle import (  # noqa: F401
     NODE_DTYPE,
