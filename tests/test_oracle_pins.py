@@ -15,7 +15,8 @@ swapped operand, a wrong child index) makes it fail:
   * degenerate rows: p = q, one-hot q, disjoint supports;
   * decisions agree with the reported acceptance probabilities; the inverse
     CDF walks ids in ascending order with the stated edge convention;
-  * an end-to-end Monte-Carlo run of draft + verify over random uniforms.
+  * an end-to-end Monte-Carlo run of draft + verify over random uniforms;
+  * the reported margins: a uniform moved by less than its margin keeps the outcome, by more changes it.
 """
 import os
 
@@ -489,3 +490,57 @@ def test_tree_walk():
     w = oracle.walk(acc, np.array([[5, 6, 7]], np.int32), 4, child=child)
     np.testing.assert_array_equal(w["path_nodes"], [[0, 1, 2, -1]])
     np.testing.assert_array_equal(w["n_accepted"], [3])
+
+
+@pytest.mark.parametrize("method", ["spechub", "rrs", "rrsw"])
+def test_margins_are_the_distance_to_the_point_where_the_outcome_changes(method):
+    """margin[] is what the parity checker's near-threshold rule rests on.  Pinned by behaviour: moving
+    a uniform by a little less than its margin never changes the outcome of that test or draw, moving
+    it by a little more (towards the threshold) does."""
+    rng = np.random.default_rng(77)
+    flips = holds = 0
+    for _ in range(200):
+        V = int(rng.integers(3, 9))
+        p, q = random_simplex(rng, V), random_simplex(rng, V)
+        a = int(np.argmax(q))
+        if method == "spechub":
+            x = int(rng.choice([y for y in range(V) if y != a]))
+            x1, x2 = (x, a) if rng.random() < 0.5 else (a, x)
+            run = lambda r1, r2, u: oracle.spechub_verify(p, q, a, x1, x2, r1, r2, u)
+        else:
+            x1, x2 = int(rng.integers(V)), int(rng.integers(V))
+            if method == "rrsw" and x2 == x1:
+                x2 = (x1 + 1) % V
+            run = lambda r1, r2, u: oracle.rrs_verify(p, q, x1, x2, r1, r2, u, method == "rrsw")
+        r = [float(rng.random()), float(rng.random()), float(rng.random())]
+        o = run(*r)
+        # uniform i decides test 1, test 2 (if performed), the residual draw (if both rejected)
+        for i in range(3):
+            m = float(o["margin"][i])
+            if not np.isfinite(m) or m <= 1e-9 or m >= 0.5:
+                continue
+            for sign in (+1, -1):
+                for scale, must_hold in ((1 - 1e-6, True), (1 + 1e-6, False)):
+                    rr = list(r)
+                    rr[i] = r[i] + sign * m * scale
+                    if not 0.0 <= rr[i] < 1.0:
+                        continue
+                    o2 = run(*rr)
+                    same = (o2["accept_idx"] == o["accept_idx"] and o2["token"] == o["token"])
+                    if must_hold:
+                        assert same, (method, i, sign, r, m)
+                        holds += 1
+                    elif not same:
+                        flips += 1
+            # beyond the margin, on one of the two sides, the outcome does change
+            changed = False
+            for sign in (+1, -1):
+                v = r[i] + sign * m * (1 + 1e-6)
+                if 0.0 <= v < 1.0:
+                    rr = list(r); rr[i] = v
+                    o2 = run(*rr)
+                    changed |= not (o2["accept_idx"] == o["accept_idx"] and o2["token"] == o["token"])
+                else:
+                    changed = True   # the threshold lies outside [0, 1) on that side: nothing to cross
+            assert changed, (method, i, r, m, dict(acc=int(o["accept_idx"]), tok=int(o["token"])))
+    assert holds > 120 and flips > 60
