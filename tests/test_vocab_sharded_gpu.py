@@ -188,3 +188,50 @@ def test_shard_argument_errors(sh):
     for bad in (vs.Shard(2, 2, 0, 128), vs.Shard(0, 65, 0, 128), vs.Shard(0, 2, 100, 128), vs.Shard(0, 1, -1, 64)):
         with pytest.raises(sh.SpecHubError):
             vs.ShardedDraft(tq, un, tree, bad, 1.0).stats()
+
+
+def test_sharded_drivers_on_a_stream_that_is_not_current(sh):
+    """The torch.distributed drivers mix launches, allocations and collectives; a caller's stream must
+    carry all of them.  One rank (NCCL, world size 1) holding the whole vocabulary: the results on a
+    side stream equal those on the current stream, and those of the plain calls."""
+    import os
+    import socket
+
+    import torch.distributed as dist
+
+    from paper_2411_05289_b200 import vocab_sharded as vs
+
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        lp, lq, un = make_case(9001, "bf16", 5)
+        tp, tq = workloads.to_device(lp, "bf16"), workloads.to_device(lq, "bf16")
+        und = torch.from_numpy(un).cuda()
+        tree = sh.Tree.heap(7)
+        shard, _ = vs.even_shards(9001, 1)[0]
+        T = torch.tensor([1.0, 0.7, 1.3, 0.9], device="cuda")
+        ref_d = vs.spechub_draft_sample_sharded(tq, und, tree, shard, T)
+        ref_v = vs.spechub_verify_tree_sharded(tp, tq, ref_d["tokens"], und, tree, shard, T)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        for rep in range(3):
+            d = vs.spechub_draft_sample_sharded(tq, und, tree, shard, T, stream=side)
+            v = vs.spechub_verify_tree_sharded(tp, tq, d["tokens"], und, tree, shard, T, stream=side)
+        side.synchronize()
+        assert torch.equal(d["tokens"], ref_d["tokens"])
+        for k in ("accept_idx", "token", "n_accepted", "n_emitted", "path_tokens"):
+            assert torch.equal(v[k], ref_v[k]), k
+        # the plain calls with an explicit stream and a per-sequence temperature tensor (a temporary of the call)
+        for rep in range(3):
+            pd = sh.spechub_draft_sample(tq, und, tree, T.double(), stream=side)
+            pv = sh.spechub_verify_tree(tp, tq, pd["tokens"], und, tree, T.double(), stream=side)
+        side.synchronize()
+        cur = sh.spechub_verify_tree(tp, tq, sh.spechub_draft_sample(tq, und, tree, T)["tokens"], und, tree, T)
+        torch.cuda.synchronize()
+        for k in ("accept_idx", "token", "n_emitted"):
+            assert torch.equal(pv[k], cur[k]), k
+    finally:
+        dist.destroy_process_group()
