@@ -656,7 +656,10 @@ def main():
         if not args.no_cpu_baseline and world == 1:
             v, desc, _ = oracle_sample(cfg, args.layout, args.cpu_seconds)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
-            line["cpu_baseline_all_cores"] = oracle_all_cores(cfg, args.layout, v, args.cpu_seconds)
+            try:
+                line["cpu_baseline_all_cores"] = oracle_all_cores(cfg, args.layout, v, args.cpu_seconds)
+            except Exception as exc:   # reported, never fatal: the single-core baseline above stands
+                line["cpu_baseline_all_cores"] = {"unavailable": str(exc).splitlines()[0][:160] if str(exc) else repr(exc)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -32,12 +32,16 @@ def _work(job):
     from . import oracle as orc   # in the worker: the plain sequential oracle
 
     kind, method, names, shape, b0, b1, temps, tokens, uniforms, node_kind = job
-    shms, arrs = zip(*[_attach(nm, shape) for nm in names])
+    if shape is None:            # no shared memory on this host: the rows came with the job
+        shms, arrs = [], list(names)
+    else:
+        shms, arrs = zip(*[_attach(nm, shape) for nm in names])
+        arrs = [a[b0:b1] for a in arrs]
     try:
         if kind == "draft":
-            out = orc.draft_batch(method, arrs[0][b0:b1], temps, uniforms)
+            out = orc.draft_batch(method, arrs[0], temps, uniforms)
         else:
-            out = orc.verify_batch(method, arrs[0][b0:b1], arrs[1][b0:b1], temps, tokens, uniforms, node_kind)
+            out = orc.verify_batch(method, arrs[0], arrs[1], temps, tokens, uniforms, node_kind)
     finally:
         del arrs
         for s in shms:
@@ -64,11 +68,17 @@ class Pool:
 
     def _share(self, arrays):
         shms = []
-        for a in arrays:
-            a = np.ascontiguousarray(a, np.float32)
-            shm = shared_memory.SharedMemory(create=True, size=max(a.nbytes, 1))
-            np.ndarray(a.shape, np.float32, buffer=shm.buf)[...] = a
-            shms.append(shm)
+        try:
+            for a in arrays:
+                a = np.ascontiguousarray(a, np.float32)
+                shm = shared_memory.SharedMemory(create=True, size=max(a.nbytes, 1))
+                shms.append(shm)
+                np.ndarray(a.shape, np.float32, buffer=shm.buf)[...] = a
+        except (OSError, ValueError) as exc:
+            for s in shms:
+                s.close()
+                s.unlink()
+            raise OSError(str(exc))
         return shms
 
     def _ranges(self, B):
@@ -79,7 +89,15 @@ class Pool:
         B = logits[0].shape[0]
         t = np.asarray(temps, np.float32)
         t = np.full(B, float(t), np.float32) if t.ndim == 0 else t
-        shms = self._share(logits)
+        try:
+            shms = self._share(logits)
+        except OSError:          # /dev/shm missing or too small: hand the rows over with the jobs instead
+            shms = None
+        if shms is None:
+            jobs = [(kind, method, [np.ascontiguousarray(a[b0:b1], np.float32) for a in logits], None, b0, b1,
+                     t[b0:b1], None if tokens is None else tokens[b0:b1], uniforms[b0:b1], node_kind)
+                    for b0, b1 in self._ranges(B)]
+            return self._pool.map(_work, jobs)
         try:
             jobs = [(kind, method, [s.name for s in shms], logits[0].shape, b0, b1, t[b0:b1],
                      None if tokens is None else tokens[b0:b1], uniforms[b0:b1], node_kind)

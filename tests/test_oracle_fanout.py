@@ -23,3 +23,18 @@ def test_fanout_equals_sequential():
             v_seq = oracle.verify_batch(m, lp, lq, T, d_seq["tokens"], un, kind)
             v_par = pool.verify_batch(m, lp, lq, T, d_seq["tokens"], un, kind)
             assert v_seq.tobytes() == v_par.tobytes()
+
+
+def test_fanout_without_shared_memory(monkeypatch):
+    """Hosts whose /dev/shm is missing or small: the rows travel with the jobs, same results."""
+    rng = np.random.default_rng(6)
+    lq = rng.normal(0, 2, (5, 2, 64)).astype(np.float32)
+    un = rng.random((5, 2, 5)).astype(np.float32)
+    with fanout.Pool(2) as pool:
+        def no_shm(arrays):
+            raise OSError("no shared memory here")
+        monkeypatch.setattr(pool, "_share", no_shm)
+        d = pool.draft_batch("spechub", lq, 1.0, un)
+    ref = oracle.draft_batch("spechub", lq, 1.0, un)
+    for k in ref:
+        np.testing.assert_array_equal(ref[k], d[k])
