@@ -542,30 +542,33 @@ def main():
     # parallel LM head): every rank holds an id range of the same rows, runs the phase kernels on its own
     # slice and exchanges 32 bytes per row between them (two all-gathers and one maximum per call over
     # NCCL; no kernel is given a peer's memory).  Reported beside the batch-sharded headline.
-    vs_ms = None
+    vs_ms, vs_err = None, None
     if world > 1:
-        from paper_2411_05289_b200 import vocab_sharded as vsh
+        try:
+            from paper_2411_05289_b200 import vocab_sharded as vsh
 
-        ctp, ctq = workloads.device_logits(cfg, device=dev)      # the common rows: same seed on every rank
-        cun = workloads.device_uniforms(cfg, device=dev)
-        shard, sp = vsh.slice_of_rank(ctp, rank, world)
-        _, sq = vsh.slice_of_rank(ctq, rank, world)
-        del ctp, ctq
+            ctp, ctq = workloads.device_logits(cfg, device=dev)      # the common rows: same seed on every rank
+            cun = workloads.device_uniforms(cfg, device=dev)
+            shard, sp = vsh.slice_of_rank(ctp, rank, world)
+            _, sq = vsh.slice_of_rank(ctq, rank, world)
+            del ctp, ctq
 
-        def vs_step():
-            d = vsh.spechub_draft_sample_sharded(sq, cun, tree, shard, cfg.temperature)
-            return vsh.spechub_verify_tree_sharded(sp, sq, d["tokens"], cun, tree, shard, cfg.temperature)
+            def vs_step():
+                d = vsh.spechub_draft_sample_sharded(sq, cun, tree, shard, cfg.temperature)
+                return vsh.spechub_verify_tree_sharded(sp, sq, d["tokens"], cun, tree, shard, cfg.temperature)
 
-        for _ in range(3):
-            vs_step()
-        barrier()
-        q0.record(stream)
-        for _ in range(args.steps):
-            vs_step()
-        q1.record(stream)
-        barrier()
-        vs_ms = q0.elapsed_time(q1) / args.steps
-        del sp, sq
+            for _ in range(3):
+                vs_step()
+            barrier()
+            q0.record(stream)
+            for _ in range(args.steps):
+                vs_step()
+            q1.record(stream)
+            barrier()
+            vs_ms = q0.elapsed_time(q1) / args.steps
+            del sp, sq
+        except Exception as exc:   # every rank runs the same code on the same shapes: a failure is common to all
+            vs_err = str(exc).splitlines()[0][:160] if str(exc) else repr(exc)
 
     tms = torch.tensor([ms, e2e_s * 1e3, verify_ms, vs_ms or 0.0], device=dev, dtype=torch.float64)
     if world > 1:
@@ -639,7 +642,7 @@ def main():
                     "nodes_per_s": (len(METHODS) * B * N / (graph_ms * 1e-3)) if graph_ms else None,
                     "note": graph_note},
                 "three_drafts_per_node": kary,
-                "vocab_sharded_step": None if world == 1 else {
+                "vocab_sharded_step": None if world == 1 else {"unavailable": vs_err} if not vs_ms else {
                     "ms_per_step": vs_ms, "nodes_per_s": B * N / (vs_ms * 1e-3), "ranks": world,
                     "nccl_version": ".".join(str(v) for v in torch.cuda.nccl.version()),
                     "note": "SpecHub draft + verify + walk of ONE batch of %d sequences whose vocabulary is sharded "
