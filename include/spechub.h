@@ -83,11 +83,13 @@ extern "C" {
 #define SPECHUB_ST_DEGENERATE_Q 4u    /* draft mass outside the excluded token is 0 (one-hot q)    */
 #define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
 #define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
-#define SPECHUB_ST_INTERNAL 32u       /* reserved: no kernel of this version waits on anything that can time out */
+#define SPECHUB_ST_INTERNAL 32u       /* a bulk copy into shared memory did not arrive within the kernel's bounded wait */
 
 /* descriptor flags: how many CTAs of a thread-block cluster share one row in the large-vocabulary
  * bf16 kernels (a tuning hint; results do not depend on it beyond fp32 summation order).  At most
- * one of the three may be set; none = the library chooses. */
+ * one of the three may be set; none = the library chooses: one CTA per row, and for RRS / RRSw the
+ * verification passes read the rows through per-warp rings of bulk copies into shared memory
+ * (cp.async.bulk) -- same results, bit for bit, as SPECHUB_FLAG_SPLIT_1, whose loads go to registers. */
 #define SPECHUB_FLAG_SPLIT_1 1u
 #define SPECHUB_FLAG_SPLIT_2 2u
 #define SPECHUB_FLAG_SPLIT_4 4u

@@ -79,12 +79,17 @@ constexpr int kLeanThreads = 256;  // 4 CTAs per SM measured best (256/512/1024:
 // CTAs per row.  With 4 CTAs per SM and 148 SMs, 592/CS rows are between their first and second
 // read at any time; at CS = 4 on V = 128256 that fits L2 (DRAM reads drop from 2.0x to 1.0x the
 // algorithmic bytes) but the per-CTA fixed work grows 4x, and the two cancel (1.6 vs 1.8 ms).
+// 0 = no flag: one CTA per row (measured on B200: the per-CTA fixed work of a split row still outweighs
+// the L2 hits), and the verification of RRS / RRSw takes its vectors from per-warp rings of bulk copies.
 int lean_split(const spechub_desc *d) {
     if (d->flags & SPECHUB_FLAG_SPLIT_1) return 1;
     if (d->flags & SPECHUB_FLAG_SPLIT_2) return 2;
     if (d->flags & SPECHUB_FLAG_SPLIT_4) return 4;
-    return 1;  // measured on B200: the per-CTA fixed work of a split row still outweighs the L2 hits
+    return 0;
 }
+
+constexpr int kMaxDevices = 64;
+std::mutex g_attr_mutex;
 
 template <class K, class... Args>
 int launch_group(K kern, int cs, unsigned rows, cudaStream_t s, Args... args) {
@@ -113,6 +118,28 @@ int launch_lean_leaf(const RowArgs &a, const NodeOutPtrs *outs, int n_out, unsig
     return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
 }
 
+// One CTA per row, the passes fed by per-warp rings of bulk copies (spechub_ring.cuh).
+template <int METHOD>
+int launch_lean_verify_ring(const RowArgs &a, unsigned rows, cudaStream_t s) {
+    auto kern = lean_verify_kernel<METHOD, kLeanThreads, 1, true>;
+    constexpr int smem = kLeanThreads / 32 * kRingWarpBytes;
+    static bool configured[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECHUB_ERR_LAUNCH;
+    {
+        std::lock_guard<std::mutex> lock(g_attr_mutex);
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+                cudaGetLastError();
+                return SPECHUB_ERR_LAUNCH;
+            }
+            configured[dev] = true;
+        }
+    }
+    kern<<<rows, kLeanThreads, smem, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+}
+
 int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_lean_verify_cs<4>(method, a, rows, s);
     if (cs == 2) return launch_lean_verify_cs<2>(method, a, rows, s);
@@ -121,12 +148,14 @@ int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cuda
         const int lrc = launch_lean_leaf(a, &o, 1, rows, s);
         if (lrc != SPECHUB_OK) return lrc;
     }
-    return launch_lean_verify_cs<1>(method, a, rows, s);
+    if (cs == 1 || method == kSpecHub) return launch_lean_verify_cs<1>(method, a, rows, s);
+    if (method == kRRS) return launch_lean_verify_ring<kRRS>(a, rows, s);
+    return launch_lean_verify_ring<kRRSw>(a, rows, s);
 }
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
     if (cs == 2) return launch_group(lean_draft_kernel<kLeanThreads, 2>, 2, rows, s, a, method);
-    // one CTA per row: 128 threads, 8 CTAs per SM measured best for the single-pass draft step
+    // one CTA per row (cs 0 or 1): 128 threads, 8 CTAs per SM measured best for the single-pass draft step
     // (64 / 128 / 256 / 512 threads: 0.41 / 0.36 / 0.38 / 0.52 ms on V = 128256; 0.078 / 0.081 / 0.102 /
     // 0.165 ms on V = 32000)
     lean_draft_ck_kernel<kLeanDraftThreads><<<rows, kLeanDraftThreads, 0, s>>>(a, method);
@@ -161,9 +190,6 @@ bool resident_fits(const spechub_desc *d, bool aligned, ResShape *out) {
     }
     return false;
 }
-
-constexpr int kMaxDevices = 64;
-std::mutex g_attr_mutex;
 
 template <int MASK, int CS>
 int launch_resident_one(int nb, const FusedArgs &f, unsigned rows, cudaStream_t s) {

@@ -304,7 +304,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(FusedArgs A, int32_t *hub_out,
                                                                             float *draft_prob) {
-    __shared__ LeanShared sh;
+    __shared__ LeanCkShared sh;
     const RowArgs &a = A.r;
     const long long r = blockIdx.x;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);

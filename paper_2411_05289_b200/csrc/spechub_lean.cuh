@@ -31,6 +31,7 @@
 #include "spechub.h"
 #include "spechub_common.cuh"
 #include "spechub_stream.cuh"
+#include "spechub_ring.cuh"
 
 namespace spechub {
 namespace cg = cooperative_groups;
@@ -46,10 +47,6 @@ struct LeanShared {
     float acc[8][kLeanMaxWarps];
     float mass[kLeanMaxWarps];
     float part[1024];  // sampler: per-thread block sums of the selected warp range
-    // draft step: checkpoint sums of pass A (per warp, every CK lane-iterations), their exponent
-    // references, and the masses of those sub-blocks on the row's scale
-    float cks[kLeanMaxWarps][kLeanCk], ckc[kLeanMaxWarps][kLeanCk];
-    float ckm[kLeanMaxWarps * kLeanCk];
     float tt2;
     int blk;
     int tok;
@@ -59,6 +56,12 @@ struct LeanShared {
     float x_sum[4];          // pass-B / pass-C sums of the slice
     float x_mass;            // slice mass for a draw from q without a given token
     int x_tok;               // a token drawn by this CTA
+};
+// draft step and leaf rows: also the checkpoint sums of pass A (per warp, every CK lane-iterations), their
+// exponent references, and the masses of those sub-blocks on the row's scale
+struct LeanCkShared : LeanShared {
+    float cks[kLeanMaxWarps][kLeanCk], ckc[kLeanMaxWarps][kLeanCk];
+    float ckm[kLeanMaxWarps * kLeanCk];
 };
 
 // The CTAs of one row.  CS = 1 compiles to no cluster instruction at all.
@@ -206,6 +209,55 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
             if (BOTH) b = rq[vi];
             lean_push(P, a, k);
             if (BOTH) lean_push(Q, b, k);
+        }
+    }
+}
+
+// Pass A over both rows with the vectors coming from the warp's ring (the first pass of its stream, forwards).
+__device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k, LeanAcc &P, LeanAcc &Q) {
+    P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
+    Q.m2 = 0xff80ff80u; Q.s = 0.f; Q.c = 0.f;
+    const int vi0 = R.lo + lane;
+    if (R.nc > 0) {
+        // the reference comes from the thread's first vector that holds a finite logit: nearly always the
+        // very first one, which the first chunk holds; otherwise look further in global memory
+        ring_wait(R);
+        if (vi0 < R.hi) {
+            uint4 a, b;
+            ring_load(R, 0, lane, a, b);
+            float m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
+            if (m0 > neg_inf()) P.c = shift_of(m0, k);
+            else {
+                for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
+                    const uint4 a2 = R.vp[vr];
+                    m0 = bf2_hmax(bf2max(bf2max(a2.x, a2.y), bf2max(a2.z, a2.w)));
+                    if (m0 > neg_inf()) { P.c = shift_of(m0, k); break; }
+                }
+            }
+            m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
+            if (m0 > neg_inf()) Q.c = shift_of(m0, k);
+            else {
+                for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
+                    const uint4 b2 = R.vq[vr];
+                    m0 = bf2_hmax(bf2max(bf2max(b2.x, b2.y), bf2max(b2.z, b2.w)));
+                    if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
+                }
+            }
+        }
+    }
+#pragma unroll 1
+    for (int c = 0; c < R.nc; ++c) {
+        ring_wait(R);
+        const int v0 = vi0 + c * kRingChunkVecs;
+#pragma unroll
+        for (int j = 0; j < kRingCh; ++j) {
+            uint4 x, y;
+            ring_load(R, j, lane, x, y);
+            if (j == kRingCh - 1) ring_release(R, lane);
+            if (v0 + j * 32 < R.hi) {
+                lean_push(P, x, k);
+                lean_push(Q, y, k);
+            }
         }
     }
 }
@@ -694,7 +746,7 @@ __device__ __forceinline__ void lean_pass_a_ck(const uint4 *rq, int lo, int hi, 
 // checkpoint sub-blocks.  C = the row's exponent shift.  Returns to every thread the token, -1 if
 // nothing has mass.  Called by all threads of the CTA, after the checkpoints are visible.
 __device__ int lean_ck_sample(const Geo &g, const __nv_bfloat16 *row, float k, float C, int CK, int excl,
-                              float u, LeanShared &sh) {
+                              float u, LeanCkShared &sh) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nslot = g.nwarps * kLeanCk;
     auto wf = [&](int vi, float(&w)[8]) {
@@ -797,7 +849,7 @@ struct LeafArgs {
 
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_leaf_kernel(LeafArgs A) {
-    __shared__ LeanShared sh;
+    __shared__ LeanCkShared sh;
     const RowArgs &a = A.r;
     const long long r = blockIdx.x;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
@@ -846,9 +898,17 @@ __device__ __forceinline__ void lean_terms(float ep, float eq, float rho, float 
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
-template <int METHOD, int THREADS, int CS>
+// RING (RRS and RRSw, one CTA per row): the three passes take their vectors from per-warp rings of bulk
+// copies (spechub_ring.cuh; THREADS / 32 * kRingWarpBytes of dynamic shared memory) instead of loading
+// them from global memory into registers.  Measured on V = 128256, 7936 rows: RRS 1.89 -> 1.72 ms, RRSw
+// 1.99 -> 1.86 ms; SpecHub's two passes gain nothing from it (1.38 -> 1.38 .. 1.44 ms: the bookkeeping of
+// the ring costs the issue slots that its pass B is short of), so SpecHub keeps the register-fed loops.
+template <int METHOD, int THREADS, int CS, bool RING = false>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(RowArgs a) {
+    static_assert(!RING || (CS == 1 && METHOD != kSpecHub), "the ring-fed form: whole rows, RRS and RRSw");
     __shared__ LeanShared sh;
+    extern __shared__ __align__(128) unsigned char ring_mem[];
+    __shared__ __align__(8) uint64_t ring_bars[RING ? THREADS / 32 : 1][kRingStages];
     const int me = RowGroup<CS>::rank();
     const long long r = blockIdx.x / CS;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
@@ -876,8 +936,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     // a flagged row, the CTA that draws for a residual / leaf token.
     bool token_elsewhere = false;
 
+    // the row's stream: pass A forwards, pass B backwards, (RRS, RRSw) pass C forwards
+    WarpRing R;
+    if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, lane);
     LeanAcc tp, tq;
-    if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
+    if (RING) lean_pass_a_ring(R, lane, k, tp, tq);
+    else if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true, METHOD == kRRS>(vp, vq, lo, hi, lane, k, tp, tq);
     {
         ArgMaxSum Ps, Qs;
@@ -943,13 +1007,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             F2 s1 = f2_make(0.f, 0.f), s2 = s1, rr = s1;
             const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ);
             const F2 nrho2 = f2_make(-rho, -rho), ncrho2 = f2_make(-crho, -crho);
-            // software pipeline: the next vector pair is in registers before this one is consumed
-            uint4 np = make_uint4(0, 0, 0, 0), nq = np;
-            if (last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
-#pragma unroll 1
-            for (int vi = last_vi; vi >= lo; vi -= 32) {
-                const uint4 cp = np, cq = nq;
-                if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
+            auto vec_b = [&](int vi, const uint4 &cp, const uint4 &cq) {
                 unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
                 if (vi == hubvec) {   // the hub's own pair is no part of the sums over y != a: -inf, mass 0
 #pragma unroll
@@ -972,6 +1030,17 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     s1 = f2_add(s1, f2_sub(m, d));            // max(-d, 0) = max(d, 0) - d, exactly
                     s2 = f2_add(s2, f2_sub(w, t));
                     rr = f2_add(rr, w);
+                }
+            };
+            {
+                // software pipeline: the next vector pair is in registers before this one is consumed
+                uint4 np = make_uint4(0, 0, 0, 0), nq = np;
+                if (last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
+#pragma unroll 1
+                for (int vi = last_vi; vi >= lo; vi -= 32) {
+                    const uint4 cp = np, cq = nq;
+                    if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
+                    vec_b(vi, cp, cq);
                 }
             }
             float s1a, s1b, s2a, s2b, ra, rb;
@@ -1049,17 +1118,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             // RRSw: the next vector pair is loaded before the current one is consumed (measured:
             // 2.21 -> 2.03 ms on V = 128256; for RRS the plain loop unrolled twice is the faster one)
             constexpr bool PIPE = (METHOD == kRRSw);
-            uint4 np = make_uint4(0, 0, 0, 0), nq = np;
-            if (PIPE && last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
-#pragma unroll(PIPE ? 1 : 2)
-            for (int vi = last_vi; vi >= lo; vi -= 32) {
-                uint4 cp, cq;
-                if (PIPE) {
-                    cp = np; cq = nq;
-                    if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
-                } else {
-                    cp = vp[vi]; cq = vq[vi];
-                }
+            auto vec_b = [&](int vi, const uint4 &cp, const uint4 &cq) {
                 const unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
                 F2 eq[4];   // e_q of the vector, by words
 #pragma unroll
@@ -1079,6 +1138,34 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     dna += (qq[0] + qq[1]) + (qq[2] + qq[3]);
                     dnb += (qq[4] + qq[5]) + (qq[6] + qq[7]);
                 }
+            };
+            uint4 np = make_uint4(0, 0, 0, 0), nq = np;
+            if (RING) {
+#pragma unroll 1
+                for (int c = R.nc - 1; c >= 0; --c) {
+                    ring_wait(R);
+                    const int v0 = lo + lane + c * kRingChunkVecs;
+#pragma unroll
+                    for (int j = kRingCh - 1; j >= 0; --j) {
+                        uint4 x, y;
+                        ring_load(R, j, lane, x, y);
+                        if (j == 0) ring_release(R, lane);
+                        if (v0 + j * 32 < hi) vec_b(v0 + j * 32, x, y);
+                    }
+                }
+            } else {
+                if (PIPE && last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
+#pragma unroll(PIPE ? 1 : 2)
+                for (int vi = last_vi; vi >= lo; vi -= 32) {
+                    uint4 cp, cq;
+                    if (PIPE) {
+                        cp = np; cq = nq;
+                        if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
+                    } else {
+                        cp = vp[vi]; cq = vq[vi];
+                    }
+                    vec_b(vi, cp, cq);
+                }
             }
             float a1a, a1b;
             f2_get(a1, a1a, a1b);
@@ -1093,16 +1180,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             // pass C: mass of the residual after two rejections
             F2 w2 = f2_make(0.f, 0.f);
             const F2 nsc2 = f2_make(-A1grho, -A1grho);
-            if (PIPE && lo + lane < hi) { np = vp[lo + lane]; nq = vq[lo + lane]; }
-#pragma unroll(PIPE ? 1 : 2)
-            for (int vi = lo + lane; vi < hi; vi += 32) {
-                uint4 cp, cq;
-                if (PIPE) {
-                    cp = np; cq = nq;
-                    if (vi + 32 < hi) { np = vp[vi + 32]; nq = vq[vi + 32]; }
-                } else {
-                    cp = vp[vi]; cq = vq[vi];
-                }
+            auto vec_c = [&](int vi, const uint4 &cp, const uint4 &cq) {
                 const unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
                 const bool x1here = (METHOD == kRRSw && vi == x1vec);
 #pragma unroll
@@ -1112,6 +1190,33 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     const F2 eq = f2_exp_word(wqs[i], k2, ncq2);
                     const F2 m = f2_max0(f2_fma(nrho2, eq, f2_exp_word(wps[i], k2, ncp2)));
                     w2 = f2_add(w2, f2_max0(f2_fma(nsc, eq, m)));
+                }
+            };
+            if (RING) {
+#pragma unroll 1
+                for (int c = 0; c < R.nc; ++c) {
+                    ring_wait(R);
+                    const int v0 = lo + lane + c * kRingChunkVecs;
+#pragma unroll
+                    for (int j = 0; j < kRingCh; ++j) {
+                        uint4 x, y;
+                        ring_load(R, j, lane, x, y);
+                        if (j == kRingCh - 1) ring_release(R, lane);
+                        if (v0 + j * 32 < hi) vec_c(v0 + j * 32, x, y);
+                    }
+                }
+            } else {
+                if (PIPE && lo + lane < hi) { np = vp[lo + lane]; nq = vq[lo + lane]; }
+#pragma unroll(PIPE ? 1 : 2)
+                for (int vi = lo + lane; vi < hi; vi += 32) {
+                    uint4 cp, cq;
+                    if (PIPE) {
+                        cp = np; cq = nq;
+                        if (vi + 32 < hi) { np = vp[vi + 32]; nq = vq[vi + 32]; }
+                    } else {
+                        cp = vp[vi]; cq = vq[vi];
+                    }
+                    vec_c(vi, cp, cq);
                 }
             }
             float w2a, w2b;
@@ -1164,6 +1269,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
         }
     } while (false);
+    if (RING) {
+        // no copy may be on its way into this CTA's shared memory when it ends; a stage that never arrived
+        // (every wait is bounded) is reported with the row
+        ring_drain(R);
+        if (__syncthreads_or(R.timed_out)) o.status |= SPECHUB_ST_INTERNAL;
+    }
     if (writer) {
         a.accept_idx[r] = o.accept_idx;
         if (!token_elsewhere) a.token[r] = o.token;
@@ -1298,7 +1409,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
 // ------------------------------------------------------------------------------------------------
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(RowArgs a, int method) {
-    __shared__ LeanShared sh;
+    __shared__ LeanCkShared sh;
     const long long r = blockIdx.x;
     const int b = static_cast<int>(r / a.nodes), n = static_cast<int>(r % a.nodes);
     const __nv_bfloat16 *rowq = static_cast<const __nv_bfloat16 *>(a.draft) + b * a.stride_seq + n * a.stride_node;

@@ -127,15 +127,16 @@ def test_small_shapes(sh, V, dtype):
     assert s.rows and s2.rows
 
 
-@pytest.mark.parametrize("split", [8, 1, 2, 4])
+@pytest.mark.parametrize("split", [0, 8, 1, 2, 4])
 @pytest.mark.parametrize("V", [4096, 8192, 9000, 12344, 16384, 16392, 24000, 32768, 40000, 65536, 70000, 81920,
                                131072, 140000, 196608, 200000, 262144, 262152])
 def test_lean_shapes(sh, V, split):
     """bf16, aligned, V % 8 == 0: shapes that take the large-vocabulary bf16 kernels (V >= 8192) or, below
     that, the general ones with ragged warp ranges.  split = 8 asks for the exponentials resident on
     chip (1, 2, 4 or 8 CTAs per row and one to four batches per lane, chosen by V; beyond 262144 ids the
-    streaming kernels); 1, 2, 4 force the two-pass streaming kernels with that many CTAs per row."""
-    if split != 8 and V > 81920:
+    streaming kernels); 1, 2, 4 force the streaming kernels with that many CTAs per row, their loads going
+    to registers; 0 is the library's choice: one CTA per row, RRS / RRSw fed by rings of bulk copies."""
+    if split not in (0, 8) and V > 81920:
         pytest.skip("the forced-split streaming kernels are covered up to 81920")
     rng = np.random.default_rng(V + 3)
     B, N = 5, 7
