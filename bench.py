@@ -64,6 +64,9 @@ def parse():
                     help="large-vocabulary verification kernels: the library's choice, the two-pass streaming "
                          "kernels (one CTA per row, or a row split over 2 / 4 CTAs), or the kernels that keep the "
                          "exponentials on chip")
+    ap.add_argument("--draft-stats", default="on", choices=["on", "off"],
+                    help="on: the step goes through the *_stats entry points (the draft call hands its per-row "
+                         "statistics of the draft logits to the verification call); off: the plain entry points")
     ap.add_argument("--kary-leg", action="store_true",
                     help="also time RRS / RRSw with three drafts per node on a ternary 40-node tree of the "
                          "workload's vocabulary (reported in breakdown, not part of `value`)")
@@ -269,7 +272,7 @@ def run_table(args):
         for layout in ("dense", "paper"):
             cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--layout", layout,
                    "--steps", str(args.steps), "--warmup", str(args.warmup), "--e2e-steps", "1",
-                   "--no-cpu-baseline", "--verify-path", args.verify_path]
+                   "--no-cpu-baseline", "--verify-path", args.verify_path, "--draft-stats", args.draft_stats]
             out = subprocess.run(cmd, capture_output=True, text=True)
             lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
             if out.returncode != 0 or not lines:
@@ -354,21 +357,34 @@ def main():
         ev_pairs.setdefault(name, []).append((e0, e1))
         return r
 
+    # The two calls of a method: with --draft-stats on (default) the draft call leaves its per-row statistics
+    # of the draft logits (16 bytes a row) for the verification call, which then reads the draft rows once
+    # instead of twice; off = the plain entry points.
+    hand_over = args.draft_stats == "on"
+
+    def do_draft(m, tq, un):
+        if m == "spechub":
+            return (sh.spechub_draft_sample_stats if hand_over else sh.spechub_draft_sample)(tq, un, tree, cfg.temperature)
+        return (sh.rrs_draft_sample_stats if hand_over else sh.rrs_draft_sample)(tq, un, tree, m == "rrsw", cfg.temperature)
+
+    def do_verify(m, tp, tq, d, un, out):
+        if m == "spechub":
+            if hand_over:
+                return sh.spechub_verify_tree_stats(tp, tq, d["stats"], d["tokens"], un, tree, cfg.temperature, out=out)
+            return sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=out)
+        if hand_over:
+            return sh.rrs_verify_tree_stats(tp, tq, d["stats"], d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=out)
+        return sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=out)
+
+    def call_name(kind, m):
+        return "spechub_%s" % kind if m == "spechub" else "rrs_%s[%s]" % (kind, m)
+
     def step(record=False):
         tp, tq, un = copies[turn[0] % len(copies)]
         turn[0] += 1
         for m in METHODS:
-            if m == "spechub":
-                d = timed("spechub_draft_sample", record,
-                          lambda: sh.spechub_draft_sample(tq, un, tree, cfg.temperature))
-                timed("spechub_verify_tree", record,
-                      lambda: sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=outs[m]))
-            else:
-                wo = m == "rrsw"
-                d = timed("rrs_draft_sample[%s]" % m, record,
-                          lambda: sh.rrs_draft_sample(tq, un, tree, wo, cfg.temperature))
-                timed("rrs_verify_tree[%s]" % m, record,
-                      lambda: sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, wo, cfg.temperature, out=outs[m]))
+            d = timed(call_name("draft_sample", m), record, lambda: do_draft(m, tq, un))
+            timed(call_name("verify_tree", m), record, lambda: do_verify(m, tp, tq, d, un, outs[m]))
 
     def barrier():
         torch.cuda.synchronize()
@@ -515,11 +531,11 @@ def main():
                 ctq.copy_(h_tq[b0:b1], non_blocking=True)
                 cun.copy_(h_un[b0:b1], non_blocking=True)
                 co = chunk_outs[ci]
-                d = sh.spechub_draft_sample(ctq, cun, tree, cfg.temperature)
-                sh.spechub_verify_tree(ctp, ctq, d["tokens"], cun, tree, cfg.temperature, out=co["spechub"])
+                d = do_draft("spechub", ctq, cun)
+                do_verify("spechub", ctp, ctq, d, cun, co["spechub"])
                 for m, wo in (("rrs", False), ("rrsw", True)):
-                    d = sh.rrs_draft_sample(ctq, cun, tree, wo, cfg.temperature)
-                    sh.rrs_verify_tree(ctp, ctq, d["tokens"], cun, tree, wo, cfg.temperature, out=co[m])
+                    d = do_draft(m, ctq, cun)
+                    do_verify(m, ctp, ctq, d, cun, co[m])
                 for m in METHODS:
                     for k in res_keys:
                         h_res[m][k][b0:b1].copy_(co[m][k], non_blocking=True)
@@ -581,8 +597,9 @@ def main():
         e2e_value = nodes_per_step * args.e2e_steps / (e2e_ms * 1e-3)
         kind = workloads.paper_node_kind(N) if args.layout == "paper" else np.zeros(N, np.uint8)
         n_leaf = int(kind.sum())
-        alg_bytes = B * ((N - n_leaf) * (2 * V * esz + 8 + 20 + 44) + n_leaf * (V * esz + 20 + 44))
-        draft_bytes = B * N * (V * esz + 8 + 8 + 16)
+        rec = 16 if hand_over else 0   # the per-row record of draft statistics: written by the draft call, read by verification
+        alg_bytes = B * ((N - n_leaf) * (2 * V * esz + 8 + 20 + 44 + rec) + n_leaf * (V * esz + 20 + 44))
+        draft_bytes = B * N * (V * esz + 8 + 8 + 16 + rec)
         peak, peak_src = measured_peak()
         total_call_ms = sum(call_ms.values())
         roof = {}
@@ -593,14 +610,17 @@ def main():
                           "frac": ach / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0,
                           "traffic": (TRAFFIC_PER_ROW[(name, args.workload)] * B * N
                                       if (name, args.workload) in TRAFFIC_PER_ROW and args.layout == "dense"
-                                      and args.verify_path == "default" else None),
+                                      and args.verify_path == "default" and hand_over else None),
                           "alg_bytes_per_launch": nbytes,
                           "ms_per_launch": t_ms, "share_of_step": t_ms / total_call_ms}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": config_dict(cfg, args.layout, world),
+            "config": dict(config_dict(cfg, args.layout, world),
+                           draft_stats=("the draft call hands max / argmax / sum of each draft row to the verification "
+                                        "call (*_stats entry points): verification's first pass reads the target row only"
+                                        if hand_over else "off: plain entry points")),
             "value_note": "each node is counted once per method (SpecHub, RRS, RRSw run one after another on the "
                           "same inputs): node-method verifications; SpecHub alone is breakdown.spechub_only_step",
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -617,10 +637,12 @@ def main():
             "roofline": roof["spechub_verify_tree"],
             "kernels": roof,
             "special_function_pipe": {
-                "note": "4 ex2 per vocabulary pair per verified row (2 in pass A, 2 in pass B); "
-                        "B200 issues 16 ex2/clk/SM (measured)",
+                "note": ("3 ex2 per vocabulary pair per verified row (1 in pass A, over the target row; 2 in pass B); "
+                         if hand_over else
+                         "4 ex2 per vocabulary pair per verified row (2 in pass A, 2 in pass B); ")
+                        + "B200 issues 16 ex2/clk/SM (measured)",
                 "kernel": "spechub_verify_tree",
-                "achieved_ex2_per_s": 4.0 * B * (N - n_leaf) * V / (verify_ms * 1e-3),
+                "achieved_ex2_per_s": (3.0 if hand_over else 4.0) * B * (N - n_leaf) * V / (verify_ms * 1e-3),
                 "peak_ex2_per_s": 148 * 16 * (clocks["sm_mhz"] or 1965.0) * 1e6,
             },
             "breakdown": {

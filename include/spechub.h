@@ -83,6 +83,7 @@ extern "C" {
 #define SPECHUB_ST_DEGENERATE_Q 4u    /* draft mass outside the excluded token is 0 (one-hot q)    */
 #define SPECHUB_ST_ZERO_MASS_DRAFT 8u /* a performed acceptance test had denominator 0: rejected   */
 #define SPECHUB_ST_ZERO_RESIDUAL 16u  /* residual mass 0 on rejection: the token was drawn from p  */
+#define SPECHUB_ST_STATS 64u          /* *_stats verification: the row's draft statistics are not those of its draft logits and temperature: output -1 */
 #define SPECHUB_ST_INTERNAL 32u       /* a bulk copy into shared memory did not arrive within the kernel's bounded wait */
 
 /* descriptor flags: how many CTAs of a thread-block cluster share one row in the large-vocabulary
@@ -209,6 +210,55 @@ int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
                         const float *uniforms, const spechub_node_out *node_out,
                         const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
                         void *stream);
+
+/*
+ * Draft statistics handed from the draft step to verification.
+ *
+ * Both steps of a decoding iteration read the same draft logits: the draft step
+ * to sample x1, x2 ~ Q (Algorithm 3; Algorithm 1 for RRS / RRSw), verification
+ * for a = argmax q, q(a) and the normaliser of q (Section 4).  The draft step
+ * knows all three once it has read the row.  spechub_draft_sample_stats /
+ * rrs_draft_sample_stats are spechub_draft_sample / rrs_draft_sample that also
+ * leave, per (sequence, node), a 16-byte record (maximum draft logit, argmax,
+ * sum of the other exponentials, a tag) in draft_stats: device memory of
+ * spechub_draft_stats_bytes(desc) bytes, 16-byte aligned, owned by the caller.
+ * spechub_verify_tree_stats / rrs_verify_tree_stats are spechub_verify_tree /
+ * rrs_verify_tree that take those records instead of making their first pass
+ * over the draft row: that pass then reads the target row only (half its
+ * bytes, half its exponentials).  Everything else -- arguments, outputs,
+ * status bits, the tree walk -- is as in the plain calls, and the results agree
+ * with theirs up to the fp32 summation order of the draft row's normaliser
+ * (accept / reject decisions can differ only where the plain call's decision
+ * is itself within rounding of its threshold).
+ *
+ * The records are opaque and tied to the library build, the descriptor (shape,
+ * strides, dtype, temperature, flags) and the draft logits they were made
+ * from; they may be used by any number of verification calls until those
+ * change.  A record that cannot be this row's -- wrong tag (other temperature
+ * or library), argmax out of range, or a draft logit at the argmax other than
+ * the recorded maximum -- flags the row SPECHUB_ST_STATS with outputs -1; other
+ * inconsistencies are the caller's responsibility.  Only the default path of
+ * the large-vocabulary bf16 shapes (no SPECHUB_FLAG_*, k = 2, rows 16-byte
+ * aligned, vocab % 8 == 0, vocab >= 8192) writes and reads records; on every
+ * other path the draft call clears draft_stats and the verification call
+ * ignores it, so the four calls may be used unconditionally.
+ */
+size_t spechub_draft_stats_bytes(const spechub_desc *desc);
+int spechub_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                               int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
+                               void *draft_stats, void *stream);
+int rrs_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                           int without_replacement, int32_t *draft_tokens, uint32_t *status,
+                           void *draft_stats, void *stream);
+int spechub_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                              const void *draft_stats, const int32_t *draft_tokens, const float *uniforms,
+                              const spechub_node_out *node_out, const spechub_seq_out *seq_out,
+                              void *workspace, size_t workspace_bytes, void *stream);
+int rrs_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                          const void *draft_stats, const int32_t *draft_tokens, const float *uniforms,
+                          int without_replacement, const spechub_node_out *node_out,
+                          const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                          void *stream);
 
 /*
  * Verification with Recursive Rejection Sampling (Algorithm 1) of every node,

@@ -17,10 +17,14 @@ from .binding import (  # noqa: F401
     mdsd_compare_draft_sample,
     mdsd_compare_verify_tree,
     rrs_draft_sample,
+    rrs_draft_sample_stats,
     rrs_verify_tree,
+    rrs_verify_tree_stats,
     set_row_split,
     spechub_draft_sample,
+    spechub_draft_sample_stats,
     spechub_verify_tree,
+    spechub_verify_tree_stats,
     spechub_verify_tree_static,
     status_string,
     workspace_bytes,

@@ -24,6 +24,8 @@ STATUS_BITS = {
     "DEGENERATE_Q": 4,
     "ZERO_MASS_DRAFT": 8,
     "ZERO_RESIDUAL": 16,
+    "INTERNAL": 32,
+    "STATS": 64,
 }
 
 
@@ -95,6 +97,20 @@ def load_library(build_if_missing: bool = True):
     lib.rrs_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, i32,
                                     ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
                                     ctypes.c_size_t, vp]
+    lib.spechub_draft_sample_stats.restype = i32
+    lib.spechub_draft_sample_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.rrs_draft_sample_stats.restype = i32
+    lib.rrs_draft_sample_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, i32, vp, vp, vp, vp]
+    lib.spechub_verify_tree_stats.restype = i32
+    lib.spechub_verify_tree_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, vp,
+                                              ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                              ctypes.c_size_t, vp]
+    lib.rrs_verify_tree_stats.restype = i32
+    lib.rrs_verify_tree_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, vp, vp, i32,
+                                          ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                          ctypes.c_size_t, vp]
+    lib.spechub_draft_stats_bytes.restype = ctypes.c_size_t
+    lib.spechub_draft_stats_bytes.argtypes = [ctypes.POINTER(_Desc)]
     lib.mdsd_compare_draft_sample.restype = i32
     lib.mdsd_compare_draft_sample.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp, vp,
                                               ctypes.POINTER(vp), vp]
@@ -289,8 +305,24 @@ def _need_k2(tree):
         raise ValueError("SpecHub takes exactly two drafts per node")
 
 
+def _alloc_stats(lib, d, dev):
+    """The caller-owned buffer of per-row draft statistics (16 bytes per row, opaque)."""
+    n = lib.spechub_draft_stats_bytes(ctypes.byref(d))
+    return torch.empty(max(n, 16) // 4, dtype=torch.int32, device=dev)
+
+
 def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
     """Draw the k = 2 SpecHub drafts of every node.  Returns dict(tokens, hub, prob, status)."""
+    return _spechub_draft(draft_logits, uniforms, tree, temperature, stream, False)
+
+
+def spechub_draft_sample_stats(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
+    """``spechub_draft_sample`` that also leaves the per-row draft statistics (key ``stats``) for
+    ``spechub_verify_tree_stats``."""
+    return _spechub_draft(draft_logits, uniforms, tree, temperature, stream, True)
+
+
+def _spechub_draft(draft_logits, uniforms, tree, temperature, stream, with_stats):
     lib = load_library()
     _need_k2(tree)
     d, keep = _desc(draft_logits, tree, temperature)
@@ -301,15 +333,33 @@ def spechub_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, st
     hub = torch.empty((B, N), dtype=torch.int32, device=dev)
     prob = torch.empty((B, N, 2), dtype=torch.float32, device=dev)
     status = torch.empty((B, N), dtype=torch.int32, device=dev)
-    _check(lib.spechub_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), _ptr(tokens),
-                                    _ptr(hub), _ptr(prob), _ptr(status), _stream_ptr(stream)))
-    _hold(keep + [tokens, hub, prob, status], stream)
-    return dict(tokens=tokens, hub=hub, prob=prob, status=status)
+    out = dict(tokens=tokens, hub=hub, prob=prob, status=status)
+    if with_stats:
+        out["stats"] = _alloc_stats(lib, d, dev)
+        _check(lib.spechub_draft_sample_stats(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), _ptr(tokens),
+                                              _ptr(hub), _ptr(prob), _ptr(status), _ptr(out["stats"]),
+                                              _stream_ptr(stream)))
+    else:
+        _check(lib.spechub_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), _ptr(tokens),
+                                        _ptr(hub), _ptr(prob), _ptr(status), _stream_ptr(stream)))
+    _hold(keep + list(out.values()), stream)
+    return out
 
 
 def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bool, temperature=1.0,
                      stream=None):
     """Draw the k = tree.k RRS / RRSw drafts of every node.  Returns dict(tokens, status)."""
+    return _rrs_draft(draft_logits, uniforms, tree, without_replacement, temperature, stream, False)
+
+
+def rrs_draft_sample_stats(draft_logits, uniforms, tree: Tree, without_replacement: bool, temperature=1.0,
+                           stream=None):
+    """``rrs_draft_sample`` that also leaves the per-row draft statistics (key ``stats``) for
+    ``rrs_verify_tree_stats``."""
+    return _rrs_draft(draft_logits, uniforms, tree, without_replacement, temperature, stream, True)
+
+
+def _rrs_draft(draft_logits, uniforms, tree, without_replacement, temperature, stream, with_stats):
     lib = load_library()
     d, keep = _desc(draft_logits, tree, temperature)
     B, N, _ = draft_logits.shape
@@ -317,11 +367,18 @@ def rrs_draft_sample(draft_logits, uniforms, tree: Tree, without_replacement: bo
     _check_uniforms(uniforms, B, N, dev, tree.k)
     tokens = torch.empty((B, N, tree.k), dtype=torch.int32, device=dev)
     status = torch.empty((B, N), dtype=torch.int32, device=dev)
-    _check(lib.rrs_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
-                                int(bool(without_replacement)), _ptr(tokens), _ptr(status),
-                                _stream_ptr(stream)))
-    _hold(keep + [tokens, status], stream)
-    return dict(tokens=tokens, status=status)
+    out = dict(tokens=tokens, status=status)
+    if with_stats:
+        out["stats"] = _alloc_stats(lib, d, dev)
+        _check(lib.rrs_draft_sample_stats(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
+                                          int(bool(without_replacement)), _ptr(tokens), _ptr(status),
+                                          _ptr(out["stats"]), _stream_ptr(stream)))
+    else:
+        _check(lib.rrs_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms),
+                                    int(bool(without_replacement)), _ptr(tokens), _ptr(status),
+                                    _stream_ptr(stream)))
+    _hold(keep + list(out.values()), stream)
+    return out
 
 
 def alloc_verify_outputs(B, N, levels, dev, k=2):
@@ -341,7 +398,7 @@ def alloc_verify_outputs(B, N, levels, dev, k=2):
 
 
 def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream,
-            out, probabilities=True):
+            out, probabilities=True, stats=None, with_stats=False):
     lib = load_library()
     _same_layout(target_logits, draft_logits)
     d, keep = _desc(target_logits, tree, temperature)
@@ -362,11 +419,21 @@ def _verify(method, target_logits, draft_logits, draft_tokens, uniforms, tree, t
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
     common = (ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms))
     tail = (ctypes.byref(no), ctypes.byref(so), _ptr(ws), ws_bytes, _stream_ptr(stream))
-    if method == "spechub":
+    if with_stats:
+        need = lib.spechub_draft_stats_bytes(ctypes.byref(d))
+        if (stats is None or stats.dtype != torch.int32 or not stats.is_contiguous() or stats.device != dev
+                or stats.numel() * 4 < need):
+            raise ValueError("stats must be the tensor a *_draft_sample_stats call returned for this shape")
+        common = common[:3] + (_ptr(stats),) + common[3:]
+        if method == "spechub":
+            _check(lib.spechub_verify_tree_stats(*common, *tail))
+        else:
+            _check(lib.rrs_verify_tree_stats(*common, 1 if method == "rrsw" else 0, *tail))
+    elif method == "spechub":
         _check(lib.spechub_verify_tree(*common, *tail))
     else:
         _check(lib.rrs_verify_tree(*common, 1 if method == "rrsw" else 0, *tail))
-    _hold(keep + [ws] + list(out.values()), stream)
+    _hold(keep + [ws, stats] + list(out.values()), stream)
     return out
 
 
@@ -385,6 +452,22 @@ def rrs_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: T
     """RRS / RRSw verification of every node and the tree walk."""
     return _verify("rrsw" if without_replacement else "rrs", target_logits, draft_logits, draft_tokens,
                    uniforms, tree, temperature, stream, out, probabilities)
+
+
+def spechub_verify_tree_stats(target_logits, draft_logits, stats, draft_tokens, uniforms, tree: Tree,
+                              temperature=1.0, stream=None, out=None, probabilities=True):
+    """``spechub_verify_tree`` given the draft statistics ``spechub_draft_sample_stats`` left for the same
+    draft logits, tree and temperature: the first pass reads the target rows only."""
+    return _verify("spechub", target_logits, draft_logits, draft_tokens, uniforms, tree, temperature,
+                   stream, out, probabilities, stats, True)
+
+
+def rrs_verify_tree_stats(target_logits, draft_logits, stats, draft_tokens, uniforms, tree: Tree,
+                          without_replacement: bool, temperature=1.0, stream=None, out=None,
+                          probabilities=True):
+    """``rrs_verify_tree`` given the draft statistics ``rrs_draft_sample_stats`` left."""
+    return _verify("rrsw" if without_replacement else "rrs", target_logits, draft_logits, draft_tokens,
+                   uniforms, tree, temperature, stream, out, probabilities, stats, True)
 
 
 METHODS = ("spechub", "rrs", "rrsw")

@@ -17,6 +17,8 @@
 #include "spechub_shard.cuh"
 #include "spechub_shard_rrs.cuh"
 
+extern "C" size_t spechub_draft_stats_bytes(const spechub_desc *desc);
+
 namespace {
 
 using namespace spechub;
@@ -119,9 +121,9 @@ int launch_lean_leaf(const RowArgs &a, const NodeOutPtrs *outs, int n_out, unsig
 }
 
 // One CTA per row, the passes fed by per-warp rings of bulk copies (spechub_ring.cuh).
-template <int METHOD>
+template <int METHOD, bool STATS>
 int launch_lean_verify_ring(const RowArgs &a, unsigned rows, cudaStream_t s) {
-    auto kern = lean_verify_kernel<METHOD, kLeanThreads, 1, true>;
+    auto kern = lean_verify_kernel<METHOD, kLeanThreads, 1, true, STATS>;
     constexpr int smem = kLeanThreads / 32 * kRingWarpBytes;
     static bool configured[kMaxDevices] = {};
     int dev = -1;
@@ -148,9 +150,17 @@ int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cuda
         const int lrc = launch_lean_leaf(a, &o, 1, rows, s);
         if (lrc != SPECHUB_OK) return lrc;
     }
+    if (cs == 0 && a.draft_stats_in) {   // the draft row's statistics come from the draft step
+        if (method == kSpecHub) {
+            lean_verify_kernel<kSpecHub, kLeanThreads, 1, false, true><<<rows, kLeanThreads, 0, s>>>(a);
+            return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
+        }
+        if (method == kRRS) return launch_lean_verify_ring<kRRS, true>(a, rows, s);
+        return launch_lean_verify_ring<kRRSw, true>(a, rows, s);
+    }
     if (cs == 1 || method == kSpecHub) return launch_lean_verify_cs<1>(method, a, rows, s);
-    if (method == kRRS) return launch_lean_verify_ring<kRRS>(a, rows, s);
-    return launch_lean_verify_ring<kRRSw>(a, rows, s);
+    if (method == kRRS) return launch_lean_verify_ring<kRRS, false>(a, rows, s);
+    return launch_lean_verify_ring<kRRSw, false>(a, rows, s);
 }
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
@@ -288,12 +298,20 @@ int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SP
 
 int draft_common(const spechub_desc *d, const void *draft_logits, const float *uniforms, int method,
                  int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
-                 void *stream) {
+                 void *stream, void *draft_stats = nullptr) {
     const int rc = check_desc(d);
     if (rc != SPECHUB_OK) return rc;
     if (d->batch == 0) return SPECHUB_OK;  // nothing to do; pointers are not looked at
     if (!draft_logits || !uniforms || !draft_tokens) return SPECHUB_ERR_NULL;
     RowArgs a = base_args(d);
+    // Only the one-CTA-per-row kernel of the large-vocabulary bf16 shapes leaves statistics; every other
+    // path leaves records that no verification accepts (tag 0), and the verification paths that pair
+    // with them do not look at the records.
+    const bool stats_kernel = d->k == 2 && lean_split(d) == 0 && lean_ok(d, rows_aligned(d, draft_logits));
+    if (draft_stats && !stats_kernel &&
+        cudaMemsetAsync(draft_stats, 0, spechub_draft_stats_bytes(d), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return SPECHUB_ERR_LAUNCH;
+    a.draft_stats_out = stats_kernel ? draft_stats : nullptr;
     a.draft = draft_logits;
     a.uniforms = uniforms;
     a.draft_tokens_out = draft_tokens;
@@ -367,7 +385,7 @@ int launch_walk(const spechub_desc *d, const spechub_node_out *no, const spechub
 int verify_common(const spechub_desc *d, const void *target_logits, const void *draft_logits,
                   const int32_t *draft_tokens, const float *uniforms, int method,
                   const spechub_node_out *no, const spechub_seq_out *so, void *workspace,
-                  size_t workspace_bytes, void *stream) {
+                  size_t workspace_bytes, void *stream, const void *draft_stats = nullptr) {
     const int rc = check_desc(d);
     if (rc != SPECHUB_OK) return rc;
     if (d->batch == 0) return SPECHUB_OK;  // nothing to do; pointers are not looked at
@@ -377,6 +395,7 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
     if (workspace_bytes < spechub_workspace_bytes(d)) return SPECHUB_ERR_WORKSPACE;
     (void)workspace;
     RowArgs a = base_args(d);
+    a.draft_stats_in = draft_stats;
     a.target = target_logits;
     a.draft = draft_logits;
     a.uniforms = uniforms;
@@ -570,6 +589,44 @@ int rrs_draft_sample(const spechub_desc *desc, const void *draft_logits, const f
                         draft_tokens, nullptr, nullptr, status, stream);
 }
 
+int spechub_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                               int32_t *draft_tokens, int32_t *hub, float *draft_prob, uint32_t *status,
+                               void *draft_stats, void *stream) {
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    return draft_common(desc, draft_logits, uniforms, kSpecHub, draft_tokens, hub, draft_prob, status,
+                        stream, draft_stats);
+}
+
+int rrs_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                           int without_replacement, int32_t *draft_tokens, uint32_t *status,
+                           void *draft_stats, void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    return draft_common(desc, draft_logits, uniforms, without_replacement ? kRRSw : kRRS,
+                        draft_tokens, nullptr, nullptr, status, stream, draft_stats);
+}
+
+int spechub_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                              const void *draft_stats, const int32_t *draft_tokens, const float *uniforms,
+                              const spechub_node_out *node_out, const spechub_seq_out *seq_out,
+                              void *workspace, size_t workspace_bytes, void *stream) {
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    return verify_common(desc, target_logits, draft_logits, draft_tokens, uniforms, kSpecHub,
+                         node_out, seq_out, workspace, workspace_bytes, stream, draft_stats);
+}
+
+int rrs_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                          const void *draft_stats, const int32_t *draft_tokens, const float *uniforms,
+                          int without_replacement, const spechub_node_out *node_out,
+                          const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                          void *stream) {
+    if (without_replacement != 0 && without_replacement != 1) return SPECHUB_ERR_METHOD;
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    return verify_common(desc, target_logits, draft_logits, draft_tokens, uniforms,
+                         without_replacement ? kRRSw : kRRS, node_out, seq_out, workspace,
+                         workspace_bytes, stream, draft_stats);
+}
+
 int spechub_verify_tree(const spechub_desc *desc, const void *target_logits,
                         const void *draft_logits, const int32_t *draft_tokens,
                         const float *uniforms, const spechub_node_out *node_out,
@@ -753,6 +810,11 @@ int rrs_shard_draft_finish(const spechub_desc *desc, const spechub_shard *shard,
 size_t spechub_workspace_bytes(const spechub_desc *desc) {
     (void)desc;
     return 0;
+}
+
+size_t spechub_draft_stats_bytes(const spechub_desc *desc) {
+    if (!desc || desc->batch < 0 || desc->nodes < 1) return 0;
+    return sizeof(DraftStat) * static_cast<size_t>(desc->batch) * static_cast<size_t>(desc->nodes);
 }
 
 const char *spechub_status_string(int code) {

@@ -56,6 +56,7 @@ struct LeanShared {
     float x_sum[4];          // pass-B / pass-C sums of the slice
     float x_mass;            // slice mass for a draw from q without a given token
     int x_tok;               // a token drawn by this CTA
+    int stat_ok;             // verification from draft statistics: the row's record was accepted
 };
 // draft step and leaf rows: also the checkpoint sums of pass A (per warp, every CK lane-iterations), their
 // exponent references, and the masses of those sub-blocks on the row's scale
@@ -214,6 +215,7 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
 }
 
 // Pass A over both rows with the vectors coming from the warp's ring (the first pass of its stream, forwards).
+template <bool BOTH>
 __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k, LeanAcc &P, LeanAcc &Q) {
     P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
     Q.m2 = 0xff80ff80u; Q.s = 0.f; Q.c = 0.f;
@@ -234,13 +236,15 @@ __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k,
                     if (m0 > neg_inf()) { P.c = shift_of(m0, k); break; }
                 }
             }
-            m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
-            if (m0 > neg_inf()) Q.c = shift_of(m0, k);
-            else {
-                for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
-                    const uint4 b2 = R.vq[vr];
-                    m0 = bf2_hmax(bf2max(bf2max(b2.x, b2.y), bf2max(b2.z, b2.w)));
-                    if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
+            if (BOTH) {
+                m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
+                if (m0 > neg_inf()) Q.c = shift_of(m0, k);
+                else {
+                    for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
+                        const uint4 b2 = R.vq[vr];
+                        m0 = bf2_hmax(bf2max(bf2max(b2.x, b2.y), bf2max(b2.z, b2.w)));
+                        if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
+                    }
                 }
             }
         }
@@ -256,7 +260,7 @@ __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k,
             if (j == kRingCh - 1) ring_release(R, lane);
             if (v0 + j * 32 < R.hi) {
                 lean_push(P, x, k);
-                lean_push(Q, y, k);
+                if (BOTH) lean_push(Q, y, k);
             }
         }
     }
@@ -903,9 +907,14 @@ __device__ __forceinline__ void lean_terms(float ep, float eq, float rho, float 
 // them from global memory into registers.  Measured on V = 128256, 7936 rows: RRS 1.89 -> 1.72 ms, RRSw
 // 1.99 -> 1.86 ms; SpecHub's two passes gain nothing from it (1.38 -> 1.38 .. 1.44 ms: the bookkeeping of
 // the ring costs the issue slots that its pass B is short of), so SpecHub keeps the register-fed loops.
-template <int METHOD, int THREADS, int CS, bool RING = false>
+// STATS (one CTA per row): the maximum, argmax and sum of the draft row come from the record the draft
+// step left (RowArgs::draft_stats_in), so pass A reads the target row only; a record that does not belong
+// to the row (tag, argmax out of range, or another logit there than the recorded maximum) flags the row
+// SPECHUB_ST_STATS.
+template <int METHOD, int THREADS, int CS, bool RING = false, bool STATS = false>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(RowArgs a) {
     static_assert(!RING || (CS == 1 && METHOD != kSpecHub), "the ring-fed form: whole rows, RRS and RRSw");
+    static_assert(!STATS || CS == 1, "draft statistics: whole rows");
     __shared__ LeanShared sh;
     extern __shared__ __align__(128) unsigned char ring_mem[];
     __shared__ __align__(8) uint64_t ring_bars[RING ? THREADS / 32 : 1][kRingStages];
@@ -938,27 +947,52 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 
     // the row's stream: pass A forwards, pass B backwards, (RRS, RRSw) pass C forwards
     WarpRing R;
-    if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, lane);
+    if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, STATS, lane);
     LeanAcc tp, tq;
-    if (RING) lean_pass_a_ring(R, lane, k, tp, tq);
-    else if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
+    if (RING) lean_pass_a_ring<!STATS>(R, lane, k, tp, tq);
+    else if (leaf || STATS) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true, METHOD == kRRS>(vp, vq, lo, hi, lane, k, tp, tq);
     {
         ArgMaxSum Ps, Qs;
-        if (leaf) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        if (leaf || STATS) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
         else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
         if (threadIdx.x == 0) {
             sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
-            sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+            if (STATS) {
+                const DraftStat ds = static_cast<const DraftStat *>(a.draft_stats_in)[r];
+                bool ok = ds.tag == (kDraftStatTag ^ __float_as_uint(k));
+                // (a record of a row without a finite maximum or sum needs no look-up: the row is flagged
+                // SPECHUB_ST_NONFINITE below, as it is without the record)
+                if (ok && ds.ml > neg_inf() && ds.ml < pinf && finite_pos(ds.sx + 1.f))
+                    ok = ds.idx >= 0 && ds.idx < a.vocab && load_one<__nv_bfloat16>(rowq, ds.idx) == ds.ml;
+                sh.stat_ok = ok;
+                sh.x_ml[1] = ds.ml; sh.x_sx[1] = ds.sx; sh.x_idx[1] = ok ? ds.idx : 0;
+            } else {
+                sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+            }
         }
     }
     RowGroup<CS>::sync();  // [1] slices published
     RowStat P, Q;
     merge_slices<CS>(sh, 0, k, P);
     merge_slices<CS>(sh, 1, k, Q);
-    const float Zp = P.sx + P.own, Zq = Q.sx + Q.own;
-    const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
-    const float rho = __fdiv_rn(Zp, Zq);
+    // (Z_p, its shift and rho change only in verification from draft statistics, when the two rows turn
+    // out to be the same row: see below)
+    float Zp = P.sx + P.own;
+    const float Zq = Q.sx + Q.own;
+    float cP = P.C, invZp = 1.f / Zp;
+    const float cQ = Q.C, invZq = 1.f / Zq;
+    float rho = __fdiv_rn(Zp, Zq);
+    // With draft statistics Z_q was summed by another kernel, in another order than Z_p here.  That is
+    // rounding, except when the target row is the draft row bit for bit: then Z_p = Z_q, every p - q is 0 and
+    // the sums S1, R, A1 are exactly 0, which a rho of 1 +- 1e-7 would turn into noise that the tests then
+    // divide by.  Pass B sees both rows and notices; the row is then redone with p's normaliser set to q's.
+    unsigned diff = 0;
+    auto rows_identical = [&]() {
+        if (__syncthreads_or(diff != 0)) return false;
+        Zp = Zq; invZp = invZq; cP = cQ; rho = 1.f;
+        return true;
+    };
     const int x1 = a.draft_tokens_in[2 * r], x2 = a.draft_tokens_in[2 * r + 1];
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
     auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
@@ -969,6 +1003,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     };
 
     do {
+        if (STATS && !sh.stat_ok) { o.status = SPECHUB_ST_STATS; break; }
         if (!(P.ml > neg_inf()) || !(P.ml < pinf) || !finite_pos(Zp)) { o.status = SPECHUB_ST_NONFINITE; break; }
         if (leaf) {
             // bonus token after the last accepted draft (Figure 2): a draw from p
@@ -985,10 +1020,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             if (!(pair_xa || pair_ax) || x < 0 || x >= a.vocab) { o.status = SPECHUB_ST_TOKEN_RANGE; break; }
             const bool degenerate = !(Q.sx > 0.f);
             const float c = degenerate ? 0.f : Q.own / Q.sx;
-            const float crho = c * rho;
+            float crho = c * rho;
             const float qa = Q.own * invZq, rest = Q.sx * invZq;
             const int hubvec = hubtok >> 3, hubel = hubtok & 7;
-            const float px = prob_p(x), qx = prob_q(x);
+            float px = prob_p(x);
+            const float qx = prob_q(x);
             if (!a.beta && !a.rate) {
                 // No probability is asked for: the first test needs scalars only, and if it accepts
                 // the transport sums decide nothing.
@@ -1004,10 +1040,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
             // pass B: S1, S2, R over ids != a (Section 4, Appendix B.1)
             // (packed: the low lane takes the even ids of a vector, the high lane the odd ones)
-            F2 s1 = f2_make(0.f, 0.f), s2 = s1, rr = s1;
+            F2 s1, s2, rr;
+            auto pass_b = [&]() {
+            s1 = s2 = rr = f2_make(0.f, 0.f);
             const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ);
             const F2 nrho2 = f2_make(-rho, -rho), ncrho2 = f2_make(-crho, -crho);
             auto vec_b = [&](int vi, const uint4 &cp, const uint4 &cq) {
+                if (STATS) diff |= (cp.x ^ cq.x) | (cp.y ^ cq.y) | (cp.z ^ cq.z) | (cp.w ^ cq.w);
                 unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
                 if (vi == hubvec) {   // the hub's own pair is no part of the sums over y != a: -inf, mass 0
 #pragma unroll
@@ -1042,6 +1081,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
                     vec_b(vi, cp, cq);
                 }
+            }
+            };
+            pass_b();
+            if (STATS && rows_identical()) {
+                crho = c;
+                px = qx;
+                pass_b();
             }
             float s1a, s1b, s2a, s2b, ra, rb;
             f2_get(s1, s1a, s1b);
@@ -1112,13 +1158,15 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
             // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
             const int x1vec = x1 >> 3, x1el = x1 & 7;
-            float dna = 0.f, dnb = 0.f;
-            F2 a1 = f2_make(0.f, 0.f);   // (packed: low lane = even ids of a vector, high lane = odd ids)
-            const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ), nrho2 = f2_make(-rho, -rho);
+            float dna, dnb;
+            F2 a1;   // (packed: low lane = even ids of a vector, high lane = odd ids)
+            const F2 k2 = f2_make(k, k), ncq2 = f2_make(-cQ, -cQ);
+            F2 ncp2, nrho2;
             // RRSw: the next vector pair is loaded before the current one is consumed (measured:
             // 2.21 -> 2.03 ms on V = 128256; for RRS the plain loop unrolled twice is the faster one)
             constexpr bool PIPE = (METHOD == kRRSw);
             auto vec_b = [&](int vi, const uint4 &cp, const uint4 &cq) {
+                if (STATS) diff |= (cp.x ^ cq.x) | (cp.y ^ cq.y) | (cp.z ^ cq.z) | (cp.w ^ cq.w);
                 const unsigned wps[4] = {cp.x, cp.y, cp.z, cp.w}, wqs[4] = {cq.x, cq.y, cq.z, cq.w};
                 F2 eq[4];   // e_q of the vector, by words
 #pragma unroll
@@ -1140,7 +1188,10 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 }
             };
             uint4 np = make_uint4(0, 0, 0, 0), nq = np;
-            if (RING) {
+            auto pass_b = [&](bool from_ring) {
+            a1 = f2_make(0.f, 0.f); dna = 0.f; dnb = 0.f;
+            ncp2 = f2_make(-cP, -cP); nrho2 = f2_make(-rho, -rho);
+            if (RING && from_ring) {
 #pragma unroll 1
                 for (int c = R.nc - 1; c >= 0; --c) {
                     ring_wait(R);
@@ -1167,6 +1218,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     vec_b(vi, cp, cq);
                 }
             }
+            };
+            pass_b(true);
+            if (STATS && rows_identical()) pass_b(false);   // (the ring's next chunks are pass C's)
             float a1a, a1b;
             f2_get(a1, a1a, a1b);
             float acc[2] = {a1a + a1b, dna + dnb};
@@ -1464,6 +1518,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_ck_kernel(
         }
     }
     if (threadIdx.x == 0) {
+        if (a.draft_stats_out) {
+            DraftStat ds;
+            ds.ml = Q.ml; ds.sx = Q.sx; ds.idx = Q.idx; ds.tag = kDraftStatTag ^ __float_as_uint(k);
+            static_cast<DraftStat *>(a.draft_stats_out)[r] = ds;
+        }
         a.draft_tokens_out[2 * r] = x1;
         a.draft_tokens_out[2 * r + 1] = x2;
         if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;

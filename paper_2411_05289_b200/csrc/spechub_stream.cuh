@@ -28,7 +28,20 @@ struct RowArgs {
     float temperature;
     int nodes, vocab;
     long long stride_seq, stride_node;
+    // per-row statistics of the draft logits, handed from the draft step to verification: [B][N] DraftStat
+    void *draft_stats_out;       // draft step, may be NULL
+    const void *draft_stats_in;  // verification through a *_stats entry point
 };
+
+// What the draft step knows about a row of draft logits once it has read it, and what verification would
+// otherwise have to read the row for a second time to find out (Section 4: a = argmax q; q(a); 1 - q(a)).
+struct DraftStat {
+    float ml;       // the row's maximum logit
+    float sx;       // sum over ids != argmax of 2^(k l - k ml), k = log2(e) / T
+    int idx;        // argmax, lowest id on ties
+    unsigned tag;   // kDraftStatTag ^ bits of k: a record of another library version or temperature is refused
+};
+constexpr unsigned kDraftStatTag = 0x51a75u << 12;
 
 enum Method { kSpecHub = 0, kRRS = 1, kRRSw = 2 };
 

@@ -269,13 +269,15 @@ def temps_array(T, B):
     return np.full(B, float(t), np.float32) if t.ndim == 0 else t
 
 
-def check_verify(method, lp, lq, T, tokens, uniforms, node_kind, gpu, stats=None, label="", pool=None):
+def check_verify(method, lp, lq, T, tokens, uniforms, node_kind, gpu, stats=None, label="", pool=None,
+                 oracle_out=None):
     """All rows of a [B][N][V] problem.  gpu: dict of numpy arrays as returned by the binding.
-    pool: an oracle.fanout.Pool to run the oracle's batch call on several cores (same results)."""
+    pool: an oracle.fanout.Pool to run the oracle's batch call on several cores (same results).
+    oracle_out: the oracle's records of an earlier check of the same problem (not computed again)."""
     stats = stats or Stats()
     B, N, V = lp.shape
     t = temps_array(T, B)
-    o = (pool or oracle).verify_batch(method, lp, lq, t, tokens, uniforms, node_kind)
+    o = oracle_out if oracle_out is not None else (pool or oracle).verify_batch(method, lp, lq, t, tokens, uniforms, node_kind)
     for b in range(B):
         for n in range(N):
             g = dict(accept_idx=int(gpu["accept_idx"][b, n]), token=int(gpu["token"][b, n]),

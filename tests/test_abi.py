@@ -23,6 +23,8 @@ def test_header_declares_the_expected_entry_points():
         "spechub_shard_stats", "spechub_shard_sums", "spechub_shard_decide", "spechub_shard_draft",
         "spechub_shard_draft_finish", "spechub_verify_tree_static",
         "rrs_shard_sums", "rrs_shard_decide", "rrs_shard_draft", "rrs_shard_draft_finish",
+        "spechub_draft_stats_bytes", "spechub_draft_sample_stats", "rrs_draft_sample_stats",
+        "spechub_verify_tree_stats", "rrs_verify_tree_stats",
         "spechub_workspace_bytes", "spechub_status_string", "spechub_abi_version"])
 
 
@@ -68,6 +70,10 @@ def test_host_side_argument_checks_need_no_gpu():
     assert call(desc(batch=-1)) == -3
     assert call(desc(dtype=5)) == -4
     assert call(desc(version=2)) == -2
+    # the calls that hand draft statistics on: the record buffer is required, its size is 16 bytes a row
+    assert lib.spechub_draft_stats_bytes(ctypes.byref(desc())) == 16 * 2 * 3
+    assert lib.spechub_draft_sample_stats(ctypes.byref(desc()), fake, fake, fake, None, None, None, None, None) == -1
+    assert lib.rrs_draft_sample_stats(ctypes.byref(desc()), fake, fake, 2, fake, None, fake, None) == -9
     assert call(desc(struct_size=8)) == -2
     assert call(desc(stride_node=63)) == -5
     assert call(desc(stride_seq=100)) == -5

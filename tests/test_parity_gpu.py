@@ -64,6 +64,18 @@ def gpu_verify(sh, method, tp, tq, tok, un, tree, T, out=None):
     return sh.rrs_verify_tree(tp, tq, tok, un, tree, method == "rrsw", T, out=out)
 
 
+def gpu_draft_stats(sh, method, tq, un, tree, T):
+    if method == "spechub":
+        return sh.spechub_draft_sample_stats(tq, un, tree, T)
+    return sh.rrs_draft_sample_stats(tq, un, tree, method == "rrsw", T)
+
+
+def gpu_verify_stats(sh, method, tp, tq, stats, tok, un, tree, T, out=None):
+    if method == "spechub":
+        return sh.spechub_verify_tree_stats(tp, tq, stats, tok, un, tree, T, out=out)
+    return sh.rrs_verify_tree_stats(tp, tq, stats, tok, un, tree, method == "rrsw", T, out=out)
+
+
 def padded(x, dtype, pad_to, device="cuda"):
     """Device copy of host fp32 [B][N][V] in the storage dtype; rows padded to a multiple of
     `pad_to` elements (0 = dense rows, which are unaligned when V is odd)."""
@@ -97,6 +109,21 @@ def run_case(sh, lp, lq, dtype, T, un, paper_layout, pad_to=0, methods=METHODS, 
         for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
             np.testing.assert_array_equal(out[k], w[k], err_msg="%s walk %s" % (label, k))
         total.add(st).add(sv)
+        if tree.k == 2:
+            # the same step with the draft statistics handed from the draft call to verification: the draft
+            # call's own outputs do not change, and verification meets the same bar against the same records
+            ds = gpu_draft_stats(sh, m, tq, und, tree, Tt)
+            stats_t = ds.pop("stats")
+            ds = parity.to_numpy(ds)
+            for k in d:
+                np.testing.assert_array_equal(ds[k], d[k], err_msg="%s draft with statistics: %s" % (label, k))
+            out2 = parity.to_numpy(gpu_verify_stats(sh, m, tp, tq, stats_t, torch.from_numpy(tok).cuda(), und, tree, Tt))
+            torch.cuda.synchronize()
+            sv2, _ = parity.check_verify(m, lp, lq, T, tok, un, kind, out2, label=label + "+stats", oracle_out=ov)
+            w2 = oracle.walk(out2["accept_idx"], out2["token"], tree.levels, node_kind=kind)
+            for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+                np.testing.assert_array_equal(out2[k], w2[k], err_msg="%s+stats walk %s" % (label, k))
+            total.add(sv2)
     return total
 
 
