@@ -214,6 +214,34 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
     }
 }
 
+// Pass A over one row with four vectors per lane in flight: the next four are requested before the current
+// four are consumed.  Same vectors in the same order as lean_pass_a<false>, so the same sums.
+__device__ __forceinline__ void lean_pass_a_deep(const uint4 *rp, int lo, int hi, int lane, float k, LeanAcc &P) {
+    P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
+    for (int vr = lo + lane; vr < hi; vr += 32) {
+        const uint4 a = rp[vr];
+        const float m0 = bf2_hmax(bf2max(bf2max(a.x, a.y), bf2max(a.z, a.w)));
+        if (m0 > neg_inf()) { P.c = shift_of(m0, k); break; }
+    }
+    const int n = (hi - lo - lane + 31) >> 5;   // this lane's vectors (<= 0: none)
+    const uint4 *p = rp + lo + lane;
+    int it = 0;
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0, n3 = n0;
+    if (4 <= n) { n0 = p[0]; n1 = p[32]; n2 = p[64]; n3 = p[96]; }
+#pragma unroll 1
+    for (; it + 4 <= n; it += 4) {
+        const uint4 a0 = n0, a1 = n1, a2 = n2, a3 = n3;
+        if (it + 8 <= n) {
+            n0 = p[32 * (it + 4)]; n1 = p[32 * (it + 5)]; n2 = p[32 * (it + 6)]; n3 = p[32 * (it + 7)];
+        }
+        lean_push(P, a0, k);
+        lean_push(P, a1, k);
+        lean_push(P, a2, k);
+        lean_push(P, a3, k);
+    }
+    for (; it < n; ++it) lean_push(P, p[32 * it], k);
+}
+
 // Pass A over both rows with the vectors coming from the warp's ring (the first pass of its stream, forwards).
 template <bool BOTH>
 __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k, LeanAcc &P, LeanAcc &Q) {
@@ -950,7 +978,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, STATS, lane);
     LeanAcc tp, tq;
     if (RING) lean_pass_a_ring<!STATS>(R, lane, k, tp, tq);
-    else if (leaf || STATS) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
+    else if (STATS) lean_pass_a_deep(vp, lo, hi, lane, k, tp);
+    else if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true, METHOD == kRRS>(vp, vq, lo, hi, lane, k, tp, tq);
     {
         ArgMaxSum Ps, Qs;
