@@ -38,14 +38,15 @@ METHODS = ("spechub", "rrs", "rrsw")
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 992 (sequence, node) rows of the
 # headline shape, from an ncu capture of the kernels as they stand (the test suite checks these numbers
 # against the committed capture summary); a launch's traffic is this per row times its row count
-# (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not captured.
+# (traffic grows in proportion to the rows).  Keyed by (API call, workload); absent = not captured.  The capture
+# is of the default step (--draft-stats on, --verify-path default); any other path reports no traffic.
 TRAFFIC_PER_ROW = {
-    ("spechub_draft_sample", "c4"): 275403008.0 / 992,
-    ("spechub_verify_tree", "c4"): 939372696.0 / 992,
-    ("rrs_draft_sample[rrs]", "c4"): 278545920.0 / 992,
-    ("rrs_verify_tree[rrs]", "c4"): 1323653824.0 / 992,
-    ("rrs_draft_sample[rrsw]", "c4"): 279179008.0 / 992,
-    ("rrs_verify_tree[rrsw]", "c4"): 1332738336.0 / 992,
+    ("spechub_draft_sample", "c4"): 275593472.0 / 992,
+    ("spechub_verify_tree", "c4"): 711615768.0 / 992,
+    ("rrs_draft_sample[rrs]", "c4"): 281195008.0 / 992,
+    ("rrs_verify_tree[rrs]", "c4"): 1101473000.0 / 992,
+    ("rrs_draft_sample[rrsw]", "c4"): 279507712.0 / 992,
+    ("rrs_verify_tree[rrsw]", "c4"): 1107966824.0 / 992,
 }
 
 

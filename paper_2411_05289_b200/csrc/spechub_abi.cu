@@ -17,8 +17,6 @@
 #include "spechub_shard.cuh"
 #include "spechub_shard_rrs.cuh"
 
-extern "C" size_t spechub_draft_stats_bytes(const spechub_desc *desc);
-
 namespace {
 
 using namespace spechub;
@@ -305,13 +303,9 @@ int draft_common(const spechub_desc *d, const void *draft_logits, const float *u
     if (!draft_logits || !uniforms || !draft_tokens) return SPECHUB_ERR_NULL;
     RowArgs a = base_args(d);
     // Only the one-CTA-per-row kernel of the large-vocabulary bf16 shapes leaves statistics; every other
-    // path leaves records that no verification accepts (tag 0), and the verification paths that pair
+    // kernel leaves records that no verification accepts (all zero), and the verification paths that pair
     // with them do not look at the records.
-    const bool stats_kernel = d->k == 2 && lean_split(d) == 0 && lean_ok(d, rows_aligned(d, draft_logits));
-    if (draft_stats && !stats_kernel &&
-        cudaMemsetAsync(draft_stats, 0, spechub_draft_stats_bytes(d), static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return SPECHUB_ERR_LAUNCH;
-    a.draft_stats_out = stats_kernel ? draft_stats : nullptr;
+    a.draft_stats_out = draft_stats;
     a.draft = draft_logits;
     a.uniforms = uniforms;
     a.draft_tokens_out = draft_tokens;

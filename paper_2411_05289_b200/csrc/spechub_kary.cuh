@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(512) kary_draft_kernel(KaryArgs A) {
         }
     }
     if (threadIdx.x == 0) {
+        void_draft_stat(a, r);
         for (int i = 0; i < K; ++i) a.draft_tokens_out[K * r + i] = x[i];
         if (a.status) a.status[r] = st;
     }

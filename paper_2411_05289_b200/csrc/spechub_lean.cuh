@@ -1401,6 +1401,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_draft_kernel(Row
     uint32_t st = 0;
     const bool bad = !(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf());
     const int hubtok = bad ? -1 : Q.idx;
+    if (writer) void_draft_stat(a, r);
     if (bad) {
         if (writer) {
             a.draft_tokens_out[2 * r] = -1; a.draft_tokens_out[2 * r + 1] = -1;

@@ -42,6 +42,10 @@ struct DraftStat {
     unsigned tag;   // kDraftStatTag ^ bits of k: a record of another library version or temperature is refused
 };
 constexpr unsigned kDraftStatTag = 0x51a75u << 12;
+// a draft kernel that keeps no statistics leaves a record that no verification accepts
+__device__ __forceinline__ void void_draft_stat(const RowArgs &a, long long r) {
+    if (a.draft_stats_out) static_cast<uint4 *>(a.draft_stats_out)[r] = make_uint4(0u, 0u, 0u, 0u);
+}
 
 enum Method { kSpecHub = 0, kRRS = 1, kRRSw = 2 };
 
@@ -192,6 +196,7 @@ __global__ void __launch_bounds__(512) draft_rows_kernel(RowArgs a, int method) 
         }
     }
     if (threadIdx.x == 0) {
+        void_draft_stat(a, r);
         a.draft_tokens_out[2 * r] = x1;
         a.draft_tokens_out[2 * r + 1] = x2;
         if (a.hub) a.hub[r] = (method == kSpecHub) ? hubtok : -1;
