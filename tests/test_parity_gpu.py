@@ -418,9 +418,10 @@ def test_config2_full(sh):
         report("c2 paper=%s" % paper, s)
 
 
-def sampled_parity(sh, cfg, n_sample, layouts=(False,), extra_rows=(), pool=None):
+def sampled_parity(sh, cfg, n_sample, layouts=(False,), extra_rows=(), pool=None, with_stats=True):
     """Full-size run on device-generated inputs; oracle (on all host cores) on sampled rows, spread
-    evenly over the tree's nodes, plus `extra_rows`."""
+    evenly over the tree's nodes, plus `extra_rows`.  with_stats: the same rows also through the entry
+    points that hand the draft statistics from the draft call to verification."""
     tp, tq = workloads.device_logits(cfg)
     und = workloads.device_uniforms(cfg)
     B, N, V = tp.shape
@@ -447,17 +448,42 @@ def sampled_parity(sh, cfg, n_sample, layouts=(False,), extra_rows=(), pool=None
             tok = dn["tokens"]
             on = {k: out[k][idx_b, idx_n].cpu().numpy()[:, None] for k in
                   ("accept_idx", "token", "hub", "beta", "rate", "status")}
-            if kind is None:
-                sv, _ = parity.check_verify(m, lp, lq, cfg.temperature, tok, un, None, on, label=cfg.name, pool=pool)
-            else:
-                sv = parity.Stats()
+            records = {}   # the oracle's records of the sampled rows, kept for the second leg below
+
+            def check_rows(on, label, sv):
+                if kind is None:
+                    _, records[-1] = parity.check_verify(m, lp, lq, cfg.temperature, tok, un, None, on, stats=sv,
+                                                         label=label, pool=pool, oracle_out=records.get(-1))
+                    return
                 for leafness in (0, 1):
                     sel = np.nonzero(kind[ns] == leafness)[0]
                     if len(sel) == 0:
                         continue
                     sub = {k: v[sel] for k, v in on.items()}
-                    parity.check_verify(m, lp[sel], lq[sel], cfg.temperature, tok[sel], un[sel],
-                                        np.array([leafness], np.uint8), sub, stats=sv, label=cfg.name, pool=pool)
+                    _, records[leafness] = parity.check_verify(
+                        m, lp[sel], lq[sel], cfg.temperature, tok[sel], un[sel], np.array([leafness], np.uint8), sub,
+                        stats=sv, label=label, pool=pool, oracle_out=records.get(leafness))
+
+            sv = parity.Stats()
+            check_rows(on, cfg.name, sv)
+            if with_stats:
+                # the step as bench.py runs it by default: the draft call hands its statistics of the draft rows
+                # to verification.  Same drafts (bit for bit), same oracle records, same bar.
+                d2 = gpu_draft_stats(sh, m, tq, und, tree, cfg.temperature)
+                assert torch.equal(d2["tokens"], d["tokens"])
+                out2 = gpu_verify_stats(sh, m, tp, tq, d2["stats"], d2["tokens"], und, tree, cfg.temperature)
+                torch.cuda.synchronize()
+                assert int((out2["status"] & 3).sum()) == 0 and int((out2["status"] & (32 | 64)).sum()) == 0
+                assert float((out2["rate"].sum(-1) - 1).abs().max()) < 1e-4
+                on2 = {k: out2[k][idx_b, idx_n].cpu().numpy()[:, None] for k in
+                       ("accept_idx", "token", "hub", "beta", "rate", "status")}
+                check_rows(on2, cfg.name + "+stats", sv)
+                full2 = parity.to_numpy({k: out2[k] for k in ("accept_idx", "token", "n_accepted", "n_emitted",
+                                                              "path_nodes", "path_tokens")})
+                w2 = oracle.walk(full2["accept_idx"], full2["token"], tree.levels, node_kind=kind)
+                for k in ("n_accepted", "n_emitted", "path_nodes", "path_tokens"):
+                    np.testing.assert_array_equal(full2[k], w2[k], err_msg=k + " (+stats)")
+                del d2, out2
             # the walk, for every sequence, against the oracle's walk of the GPU's node outputs
             full = parity.to_numpy({k: out[k] for k in ("accept_idx", "token", "n_accepted", "n_emitted",
                                                         "path_nodes", "path_tokens")})
@@ -490,7 +516,7 @@ def test_config4_sampled(sh, pool, split, n_sample):
     cfg = workloads.CONFIGS["c4"]
     sh.set_row_split(split)
     try:
-        s = sampled_parity(sh, cfg, n_sample, layouts=(False, True), pool=pool)
+        s = sampled_parity(sh, cfg, n_sample, layouts=(False, True), pool=pool, with_stats=(split == 0))
     finally:
         sh.set_row_split(0)
     report("c4 split=%d" % split, s)
