@@ -216,7 +216,16 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
 
 // Pass A over one row with four vectors per lane in flight: the next four are requested before the current
 // four are consumed.  Same vectors in the same order as lean_pass_a<false>, so the same sums.
+// a 16-byte load with an L2 eviction policy (createpolicy)
+__device__ __forceinline__ uint4 ld_l2_hint(const uint4 *p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
 __device__ __forceinline__ void lean_pass_a_deep(const uint4 *rp, int lo, int hi, int lane, float k, LeanAcc &P) {
+    uint64_t pol;   // the row is read again by pass B: L2 is asked to keep it
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
     P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
     for (int vr = lo + lane; vr < hi; vr += 32) {
         const uint4 a = rp[vr];
@@ -227,12 +236,13 @@ __device__ __forceinline__ void lean_pass_a_deep(const uint4 *rp, int lo, int hi
     const uint4 *p = rp + lo + lane;
     int it = 0;
     uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0, n3 = n0;
-    if (4 <= n) { n0 = p[0]; n1 = p[32]; n2 = p[64]; n3 = p[96]; }
+    if (4 <= n) { n0 = ld_l2_hint(p, pol); n1 = ld_l2_hint(p + 32, pol); n2 = ld_l2_hint(p + 64, pol); n3 = ld_l2_hint(p + 96, pol); }
 #pragma unroll 1
     for (; it + 4 <= n; it += 4) {
         const uint4 a0 = n0, a1 = n1, a2 = n2, a3 = n3;
         if (it + 8 <= n) {
-            n0 = p[32 * (it + 4)]; n1 = p[32 * (it + 5)]; n2 = p[32 * (it + 6)]; n3 = p[32 * (it + 7)];
+            n0 = ld_l2_hint(p + 32 * (it + 4), pol); n1 = ld_l2_hint(p + 32 * (it + 5), pol);
+            n2 = ld_l2_hint(p + 32 * (it + 6), pol); n3 = ld_l2_hint(p + 32 * (it + 7), pol);
         }
         lean_push(P, a0, k);
         lean_push(P, a1, k);
@@ -1101,13 +1111,19 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                 }
             };
             {
-                // software pipeline: the next vector pair is in registers before this one is consumed
+                // software pipeline: the next vector pair is in registers before this one is consumed.
+                // From draft statistics this is the last use of both rows: the loads tell L2 to let these
+                // lines go first (and pass A told it to keep the target row's), 1.07 -> 1.02 ms on
+                // V = 128256; the kernel that reads both rows twice loses with such hints.
+                uint64_t polf = 0;
+                if (STATS) asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(polf));
+                auto ldb = [&](const uint4 *ptr) { return STATS ? ld_l2_hint(ptr, polf) : *ptr; };
                 uint4 np = make_uint4(0, 0, 0, 0), nq = np;
-                if (last_vi >= lo) { np = vp[last_vi]; nq = vq[last_vi]; }
+                if (last_vi >= lo) { np = ldb(vp + last_vi); nq = ldb(vq + last_vi); }
 #pragma unroll 1
                 for (int vi = last_vi; vi >= lo; vi -= 32) {
                     const uint4 cp = np, cq = nq;
-                    if (vi - 32 >= lo) { np = vp[vi - 32]; nq = vq[vi - 32]; }
+                    if (vi - 32 >= lo) { np = ldb(vp + vi - 32); nq = ldb(vq + vi - 32); }
                     vec_b(vi, cp, cq);
                 }
             }
