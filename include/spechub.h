@@ -66,7 +66,7 @@ extern "C" {
 #define SPECHUB_ERR_VERSION (-2)     /* struct_size / version do not match this library   */
 #define SPECHUB_ERR_SHAPE (-3)       /* batch < 0, nodes < 1, vocab < 2, k outside 2..8 (SpecHub: k != 2), levels < 1, bad flags */
 #define SPECHUB_ERR_DTYPE (-4)       /* dtype is not SPECHUB_F32 / SPECHUB_BF16            */
-#define SPECHUB_ERR_STRIDE (-5)      /* stride_node < vocab or stride_seq too small        */
+#define SPECHUB_ERR_STRIDE (-5)      /* stride_node < vocab or stride_seq too small; draft_stats not 16-byte aligned */
 #define SPECHUB_ERR_TEMPERATURE (-6) /* temperature not a finite number > 0               */
 #define SPECHUB_ERR_WORKSPACE (-7)   /* workspace smaller than spechub_workspace_bytes()   */
 #define SPECHUB_ERR_LAUNCH (-8)      /* the CUDA runtime refused a launch                  */

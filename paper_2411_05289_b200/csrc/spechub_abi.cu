@@ -301,6 +301,7 @@ int draft_common(const spechub_desc *d, const void *draft_logits, const float *u
     if (rc != SPECHUB_OK) return rc;
     if (d->batch == 0) return SPECHUB_OK;  // nothing to do; pointers are not looked at
     if (!draft_logits || !uniforms || !draft_tokens) return SPECHUB_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(draft_stats) % 16 != 0) return SPECHUB_ERR_STRIDE;
     RowArgs a = base_args(d);
     // Only the one-CTA-per-row kernel of the large-vocabulary bf16 shapes leaves statistics; every other
     // kernel leaves records that no verification accepts (all zero), and the verification paths that pair
@@ -387,6 +388,7 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
         !no->token)
         return SPECHUB_ERR_NULL;
     if (workspace_bytes < spechub_workspace_bytes(d)) return SPECHUB_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(draft_stats) % 16 != 0) return SPECHUB_ERR_STRIDE;
     (void)workspace;
     RowArgs a = base_args(d);
     a.draft_stats_in = draft_stats;

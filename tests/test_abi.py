@@ -74,6 +74,14 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.spechub_draft_stats_bytes(ctypes.byref(desc())) == 16 * 2 * 3
     assert lib.spechub_draft_sample_stats(ctypes.byref(desc()), fake, fake, fake, None, None, None, None, None) == -1
     assert lib.rrs_draft_sample_stats(ctypes.byref(desc()), fake, fake, 2, fake, None, fake, None) == -9
+    odd = ctypes.c_void_p(24)   # a record buffer that is not 16-byte aligned is refused before any launch
+    assert lib.spechub_draft_sample_stats(ctypes.byref(desc()), fake, fake, fake, None, None, None, odd, None) == -5
+    from paper_2411_05289_b200.binding import _NodeOut
+
+    no = _NodeOut(16, 16, None, None, None, None)   # (pointers never followed: the call is refused first)
+    assert lib.spechub_verify_tree_stats(ctypes.byref(desc()), fake, fake, odd, fake, fake, ctypes.byref(no), None,
+                                         None, 0, None) == -5
+
     assert call(desc(struct_size=8)) == -2
     assert call(desc(stride_node=63)) == -5
     assert call(desc(stride_seq=100)) == -5
