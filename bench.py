@@ -433,6 +433,11 @@ def main():
 
     # ---- extra: the same step through the three-method calls (shared reads of p and q) ----
     def fused_step():
+        if hand_over:
+            d = sh.mdsd_compare_draft_sample_stats(tq, un, tree, cfg.temperature)
+            sh.mdsd_compare_verify_tree_stats(tp, tq, d["stats"], {m: d[m]["tokens"] for m in METHODS}, un, tree,
+                                              cfg.temperature, out=outs)
+            return
         d = sh.mdsd_compare_draft_sample(tq, un, tree, cfg.temperature)
         sh.mdsd_compare_verify_tree(tp, tq, {m: d[m]["tokens"] for m in METHODS}, un, tree, cfg.temperature,
                                     out=outs)
@@ -673,7 +678,7 @@ def main():
                 "step_through_three_method_calls": {
                     "ms_per_step": fused_ms, "nodes_per_s": len(METHODS) * B * N / (fused_ms * 1e-3),
                     "gpu_launches_per_step": 5,
-                    "note": "mdsd_compare_draft_sample + mdsd_compare_verify_tree: same outputs as the "
+                    "note": "mdsd_compare_draft_sample + mdsd_compare_verify_tree (their _stats forms with --draft-stats on): same outputs as the "
                             "nine launches of the timed step, bit for bit; this rank only; not part of `value`"},
             },
         }

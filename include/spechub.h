@@ -316,6 +316,20 @@ int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits
                              void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The three-method calls with the hand-over of draft statistics (see
+ * spechub_draft_sample_stats): one record per row serves the three methods.
+ * Results are those of the per-method *_stats calls, bit for bit.
+ */
+int mdsd_compare_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                                    int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
+                                    uint32_t *const status[3], void *draft_stats, void *stream);
+int mdsd_compare_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                                   const void *draft_stats, const int32_t *const draft_tokens[3],
+                                   const float *uniforms, const spechub_node_out node_out[3],
+                                   const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                                   void *stream);
+
+/*
  * Tree walk alone (Figure 2) over per-node results already in device memory:
  * accept_idx, token [B][N] (in), seq_out as in spechub_verify_tree.  Used after
  * the vocabulary-sharded phases below, once the tokens have been exchanged.

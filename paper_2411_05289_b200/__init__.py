@@ -15,7 +15,9 @@ from .binding import (  # noqa: F401
     library_path,
     load_library,
     mdsd_compare_draft_sample,
+    mdsd_compare_draft_sample_stats,
     mdsd_compare_verify_tree,
+    mdsd_compare_verify_tree_stats,
     rrs_draft_sample,
     rrs_draft_sample_stats,
     rrs_verify_tree,

@@ -114,6 +114,13 @@ def load_library(build_if_missing: bool = True):
     lib.mdsd_compare_draft_sample.restype = i32
     lib.mdsd_compare_draft_sample.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp, vp,
                                               ctypes.POINTER(vp), vp]
+    lib.mdsd_compare_draft_sample_stats.restype = i32
+    lib.mdsd_compare_draft_sample_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp, vp,
+                                                    ctypes.POINTER(vp), vp, vp]
+    lib.mdsd_compare_verify_tree_stats.restype = i32
+    lib.mdsd_compare_verify_tree_stats.argtypes = [ctypes.POINTER(_Desc), vp, vp, vp, ctypes.POINTER(vp), vp,
+                                                   ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
+                                                   ctypes.c_size_t, vp]
     lib.mdsd_compare_verify_tree.restype = i32
     lib.mdsd_compare_verify_tree.argtypes = [ctypes.POINTER(_Desc), vp, vp, ctypes.POINTER(vp), vp,
                                              ctypes.POINTER(_NodeOut), ctypes.POINTER(_SeqOut), vp,
@@ -476,6 +483,16 @@ METHODS = ("spechub", "rrs", "rrsw")
 def mdsd_compare_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
     """Draft step of SpecHub, RRS and RRSw on the same q and uniforms.  Returns a dict keyed by
     method name; each entry is what the method's own draft call returns."""
+    return _compare_draft(draft_logits, uniforms, tree, temperature, stream, False)
+
+
+def mdsd_compare_draft_sample_stats(draft_logits, uniforms, tree: Tree, temperature=1.0, stream=None):
+    """``mdsd_compare_draft_sample`` that also leaves the per-row draft statistics (key ``stats`` of the
+    returned dict, one buffer for the three methods) for ``mdsd_compare_verify_tree_stats``."""
+    return _compare_draft(draft_logits, uniforms, tree, temperature, stream, True)
+
+
+def _compare_draft(draft_logits, uniforms, tree, temperature, stream, with_stats):
     lib = load_library()
     _need_k2(tree)
     d, keep = _desc(draft_logits, tree, temperature)
@@ -488,12 +505,21 @@ def mdsd_compare_draft_sample(draft_logits, uniforms, tree: Tree, temperature=1.
     prob = torch.empty((B, N, 2), dtype=torch.float32, device=dev)
     tp = (ctypes.c_void_p * 3)(*[t.data_ptr() for t in tokens])
     sp = (ctypes.c_void_p * 3)(*[t.data_ptr() for t in status])
-    _check(lib.mdsd_compare_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), tp, _ptr(hub),
-                                         _ptr(prob), sp, _stream_ptr(stream)))
-    _hold(keep + tokens + status + [hub, prob], stream)
-    return dict(spechub=dict(tokens=tokens[0], hub=hub, prob=prob, status=status[0]),
-                rrs=dict(tokens=tokens[1], status=status[1]),
-                rrsw=dict(tokens=tokens[2], status=status[2]))
+    stats = None
+    if with_stats:
+        stats = _alloc_stats(lib, d, dev)
+        _check(lib.mdsd_compare_draft_sample_stats(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), tp,
+                                                   _ptr(hub), _ptr(prob), sp, _ptr(stats), _stream_ptr(stream)))
+    else:
+        _check(lib.mdsd_compare_draft_sample(ctypes.byref(d), _ptr(draft_logits), _ptr(uniforms), tp, _ptr(hub),
+                                             _ptr(prob), sp, _stream_ptr(stream)))
+    _hold(keep + tokens + status + [hub, prob, stats], stream)
+    res = dict(spechub=dict(tokens=tokens[0], hub=hub, prob=prob, status=status[0]),
+               rrs=dict(tokens=tokens[1], status=status[1]),
+               rrsw=dict(tokens=tokens[2], status=status[2]))
+    if with_stats:
+        res["stats"] = stats
+    return res
 
 
 def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms, tree: Tree,
@@ -501,6 +527,19 @@ def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms
     """Verification and tree walk by SpecHub, RRS and RRSw from shared reads of p and q.
     ``draft_tokens`` and ``out`` are dicts keyed by method name (``out`` entries as made by
     ``alloc_verify_outputs``).  Returns ``out``."""
+    return _compare_verify(target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream, out,
+                           probabilities, None, False)
+
+
+def mdsd_compare_verify_tree_stats(target_logits, draft_logits, stats, draft_tokens, uniforms, tree: Tree,
+                                   temperature=1.0, stream=None, out=None, probabilities=True):
+    """``mdsd_compare_verify_tree`` given the draft statistics ``mdsd_compare_draft_sample_stats`` left."""
+    return _compare_verify(target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream, out,
+                           probabilities, stats, True)
+
+
+def _compare_verify(target_logits, draft_logits, draft_tokens, uniforms, tree, temperature, stream, out,
+                    probabilities, stats, with_stats):
     lib = load_library()
     _need_k2(tree)
     _same_layout(target_logits, draft_logits)
@@ -523,9 +562,18 @@ def mdsd_compare_verify_tree(target_logits, draft_logits, draft_tokens, uniforms
     tp = (ctypes.c_void_p * 3)(*[draft_tokens[m].data_ptr() for m in METHODS])
     ws_bytes = lib.spechub_workspace_bytes(ctypes.byref(d))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
-    _check(lib.mdsd_compare_verify_tree(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), tp,
-                                        _ptr(uniforms), no, so, _ptr(ws), ws_bytes, _stream_ptr(stream)))
-    _hold(keep + [ws] + [t for m in METHODS for t in out[m].values()], stream)
+    if with_stats:
+        need = lib.spechub_draft_stats_bytes(ctypes.byref(d))
+        if (stats is None or stats.dtype != torch.int32 or not stats.is_contiguous() or stats.device != dev
+                or stats.numel() * 4 < need):
+            raise ValueError("stats must be the tensor a *_draft_sample_stats call returned for this shape")
+        _check(lib.mdsd_compare_verify_tree_stats(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits),
+                                                  _ptr(stats), tp, _ptr(uniforms), no, so, _ptr(ws), ws_bytes,
+                                                  _stream_ptr(stream)))
+    else:
+        _check(lib.mdsd_compare_verify_tree(ctypes.byref(d), _ptr(target_logits), _ptr(draft_logits), tp,
+                                            _ptr(uniforms), no, so, _ptr(ws), ws_bytes, _stream_ptr(stream)))
+    _hold(keep + [ws, stats] + [t for m in METHODS for t in out[m].values()], stream)
     return out
 
 

@@ -17,6 +17,8 @@
 #include "spechub_shard.cuh"
 #include "spechub_shard_rrs.cuh"
 
+extern "C" size_t spechub_draft_stats_bytes(const spechub_desc *desc);
+
 namespace {
 
 using namespace spechub;
@@ -442,17 +444,19 @@ int verify_common(const spechub_desc *d, const void *target_logits, const void *
 // One kernel for the three methods where the lean kernels apply, the three separate paths otherwise.
 int compare_draft(const spechub_desc *d, const void *draft_logits, const float *uniforms,
                   int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
-                  uint32_t *const status[3], void *stream) {
+                  uint32_t *const status[3], void *stream, void *draft_stats = nullptr) {
     const int rc = check_desc(d);
     if (rc != SPECHUB_OK) return rc;
     if (d->k != 2) return SPECHUB_ERR_SHAPE;
     if (d->batch == 0) return SPECHUB_OK;
     if (!draft_logits || !uniforms || !draft_tokens || !draft_tokens[0] || !draft_tokens[1] || !draft_tokens[2])
         return SPECHUB_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(draft_stats) % 16 != 0) return SPECHUB_ERR_STRIDE;
     if (!lean_ok(d, rows_aligned(d, draft_logits))) {
         for (int m = 0; m < 3; ++m) {
             const int mrc = draft_common(d, draft_logits, uniforms, m, draft_tokens[m], m == 0 ? hub : nullptr,
-                                         m == 0 ? draft_prob : nullptr, status ? status[m] : nullptr, stream);
+                                         m == 0 ? draft_prob : nullptr, status ? status[m] : nullptr, stream,
+                                         m == 0 ? draft_stats : nullptr);   // (void records)
             if (mrc != SPECHUB_OK) return mrc;
         }
         return SPECHUB_OK;
@@ -461,6 +465,11 @@ int compare_draft(const spechub_desc *d, const void *draft_logits, const float *
     f.r = base_args(d);
     f.r.draft = draft_logits;
     f.r.uniforms = uniforms;
+    // records are kept where the per-method calls keep them: no split flag
+    if (draft_stats && lean_split(d) != 0 &&
+        cudaMemsetAsync(draft_stats, 0, spechub_draft_stats_bytes(d), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return SPECHUB_ERR_LAUNCH;
+    f.r.draft_stats_out = lean_split(d) == 0 ? draft_stats : nullptr;
     for (int m = 0; m < 3; ++m) {
         f.tok_out[m] = draft_tokens[m];
         f.dstatus[m] = status ? status[m] : nullptr;
@@ -474,7 +483,7 @@ int compare_draft(const spechub_desc *d, const void *draft_logits, const float *
 int compare_verify(const spechub_desc *d, const void *target_logits, const void *draft_logits,
                    const int32_t *const draft_tokens[3], const float *uniforms,
                    const spechub_node_out *no, const spechub_seq_out *so, void *workspace,
-                   size_t workspace_bytes, void *stream) {
+                   size_t workspace_bytes, void *stream, const void *draft_stats = nullptr) {
     const int rc = check_desc(d);
     if (rc != SPECHUB_OK) return rc;
     if (d->k != 2) return SPECHUB_ERR_SHAPE;
@@ -487,7 +496,7 @@ int compare_verify(const spechub_desc *d, const void *target_logits, const void 
     if (!lean_ok(d, al)) {
         for (int m = 0; m < 3; ++m) {
             const int mrc = verify_common(d, target_logits, draft_logits, draft_tokens[m], uniforms, m, &no[m],
-                                          so ? &so[m] : nullptr, workspace, workspace_bytes, stream);
+                                          so ? &so[m] : nullptr, workspace, workspace_bytes, stream, draft_stats);
             if (mrc != SPECHUB_OK) return mrc;
         }
         return SPECHUB_OK;
@@ -512,7 +521,12 @@ int compare_verify(const spechub_desc *d, const void *target_logits, const void 
             const int llrc = launch_lean_leaf(f.r, f.out, 3, rows, s);
             if (llrc != SPECHUB_OK) return llrc;
         }
-        fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
+        if (draft_stats && lean_split(d) == 0) {
+            f.r.draft_stats_in = draft_stats;
+            fused_verify_kernel<kLeanThreads, true><<<rows, kLeanThreads, 0, s>>>(f);
+        } else {
+            fused_verify_kernel<kLeanThreads><<<rows, kLeanThreads, 0, s>>>(f);
+        }
         lrc = launch_status();
     }
     for (int m = 0; m < 3 && lrc == SPECHUB_OK && so; ++m) lrc = launch_walk(d, &no[m], &so[m], s);
@@ -646,6 +660,24 @@ int mdsd_compare_draft_sample(const spechub_desc *desc, const void *draft_logits
                               int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
                               uint32_t *const status[3], void *stream) {
     return compare_draft(desc, draft_logits, uniforms, draft_tokens, hub, draft_prob, status, stream);
+}
+
+int mdsd_compare_draft_sample_stats(const spechub_desc *desc, const void *draft_logits, const float *uniforms,
+                                    int32_t *const draft_tokens[3], int32_t *hub, float *draft_prob,
+                                    uint32_t *const status[3], void *draft_stats, void *stream) {
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    return compare_draft(desc, draft_logits, uniforms, draft_tokens, hub, draft_prob, status, stream, draft_stats);
+}
+
+int mdsd_compare_verify_tree_stats(const spechub_desc *desc, const void *target_logits, const void *draft_logits,
+                                   const void *draft_stats, const int32_t *const draft_tokens[3],
+                                   const float *uniforms, const spechub_node_out node_out[3],
+                                   const spechub_seq_out *seq_out, void *workspace, size_t workspace_bytes,
+                                   void *stream) {
+    if (!draft_stats && desc && desc->batch != 0) return SPECHUB_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(draft_stats) % 16 != 0) return SPECHUB_ERR_STRIDE;
+    return compare_verify(desc, target_logits, draft_logits, draft_tokens, uniforms, node_out, seq_out,
+                          workspace, workspace_bytes, stream, draft_stats);
 }
 
 int mdsd_compare_verify_tree(const spechub_desc *desc, const void *target_logits, const void *draft_logits,

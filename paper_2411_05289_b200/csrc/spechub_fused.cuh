@@ -32,7 +32,10 @@ __device__ __forceinline__ void write_node3(const NodeOutPtrs &p, long long r, c
     if (p.status) p.status[r] = o.status;
 }
 
-template <int THREADS>
+// STATS: as in lean_verify_kernel -- the draft row's maximum, argmax and sum come from the record the draft
+// step left, pass A reads the target row only, and a row pair that turns out to be one row twice is redone
+// with p's normaliser set to q's.
+template <int THREADS, bool STATS = false>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(FusedArgs A) {
     __shared__ LeanShared sh;
     const RowArgs &a = A.r;
@@ -66,22 +69,40 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
 
     if (leaf) return;   // leaf rows belong to lean_leaf_kernel
     LeanAcc tp, tq;
-    lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
+    if (STATS) lean_pass_a_deep(vp, lo, hi, lane, k, tp);
+    else lean_pass_a<true>(vp, vq, lo, hi, lane, k, tp, tq);
     {
         ArgMaxSum Ps, Qs;
-        lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        if (STATS) lean_reduce2<false>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
+        else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
         if (t0) {
             sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
-            sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+            if (STATS) {
+                const DraftStat ds = static_cast<const DraftStat *>(a.draft_stats_in)[r];
+                bool ok = ds.tag == (kDraftStatTag ^ __float_as_uint(k));
+                if (ok && ds.ml > neg_inf() && ds.ml < pinf && finite_pos(ds.sx + 1.f))
+                    ok = ds.idx >= 0 && ds.idx < a.vocab && load_one<__nv_bfloat16>(rowq, ds.idx) == ds.ml;
+                sh.stat_ok = ok;
+                sh.x_ml[1] = ds.ml; sh.x_sx[1] = ds.sx; sh.x_idx[1] = ok ? ds.idx : 0;
+            } else {
+                sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
+            }
         }
     }
     __syncthreads();
     RowStat P, Q;
     merge_slices<1>(sh, 0, k, P);
     merge_slices<1>(sh, 1, k, Q);
-    const float Zp = P.sx + P.own, Zq = Q.sx + Q.own;
-    const float cP = P.C, cQ = Q.C, invZp = 1.f / Zp, invZq = 1.f / Zq;
-    const float rho = __fdiv_rn(Zp, Zq);
+    float Zp = P.sx + P.own;
+    const float Zq = Q.sx + Q.own;
+    float cP = P.C, invZp = 1.f / Zp;
+    const float cQ = Q.C, invZq = 1.f / Zq;
+    float rho = __fdiv_rn(Zp, Zq);
+    if (STATS && !sh.stat_ok) {
+        for (int m = 0; m < 3; ++m) o[m].status = SPECHUB_ST_STATS;
+        finish();
+        return;
+    }
     auto prob_p = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowp, y), k, cP, invZp); };
     auto prob_q = [&](int y) { return prob_of(load_one<__nv_bfloat16>(rowq, y), k, cQ, invZq); };
     auto draw_from_p = [&]() { return lean_sample_row<1>(g, rowp, k, P, 0, -1, ures, 0, sh); };
@@ -114,20 +135,25 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     if (!ok_r[1]) o[2].status = SPECHUB_ST_TOKEN_RANGE;
     const bool degenerate = !(Q.sx > 0.f);
     const float c = degenerate ? 0.f : Q.own / Q.sx;
-    const float crho = c * rho;
+    float crho = c * rho;
     const float qa = Q.own * invZq, rest = Q.sx * invZq;
     const int hubvec = hubtok >> 3, hubel = hubtok & 7;
     const int wx1 = ok_r[1] ? rx1[1] : -1;            // RRSw's first draft (left out of its renormaliser)
     const int wvec = wx1 >> 3, wel = wx1 & 7;
 
     // ---- pass B (backwards): SpecHub S1, S2, R; A1; RRSw's sum of q outside its x1 ----
-    float s1a = 0.f, s2a = 0.f, ra = 0.f, s1b = 0.f, s2b = 0.f, rb = 0.f;
-    float a1a = 0.f, a1b = 0.f, dna = 0.f, dnb = 0.f;
+    float s1a, s2a, ra, s1b, s2b, rb, a1a, a1b, dna, dnb;
+    unsigned diff = 0;
+    auto pass_b = [&]() {
+    s1a = s2a = ra = s1b = s2b = rb = 0.f;
+    a1a = a1b = dna = dnb = 0.f;
 #pragma unroll 2
     for (int vi = last_vi; vi >= lo; vi -= 32) {
         float fp[8], fq[8];
-        unpack_bf16x8(vp[vi], fp);
-        unpack_bf16x8(vq[vi], fq);
+        const uint4 rawp = vp[vi], rawq = vq[vi];
+        if (STATS) diff |= (rawp.x ^ rawq.x) | (rawp.y ^ rawq.y) | (rawp.z ^ rawq.z) | (rawp.w ^ rawq.w);
+        unpack_bf16x8(rawp, fp);
+        unpack_bf16x8(rawq, fq);
         float pp[8], qq[8];   // e_p, e_q (lean_terms: everything below is in units of 1 / Z_p)
 #pragma unroll
         for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
@@ -161,6 +187,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
             lean_terms(pp[i + 1], qq[i + 1], rho, crho, d, t);
             s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
         }
+    }
+    };
+    pass_b();
+    if (STATS && !__syncthreads_or(diff != 0)) {   // the target row is the draft row: Z_p = Z_q exactly
+        Zp = Zq; invZp = invZq; cP = cQ; rho = 1.f; crho = c;
+        pass_b();
     }
     float accB[5] = {s1a + s1b, s2a + s2b, ra + rb, a1a + a1b, dna + dnb};
     lean_block_sums<5, 0>(accB, sh);   // per-warp R stays in sh.acc[2]
@@ -330,6 +362,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_draft_kernel(Fu
     RowStat Q;
     merge_slices<1>(sh, 0, k, Q);
     const float Zq = Q.sx + Q.own;
+    if (t0 && a.draft_stats_out) {   // the record lean_draft_ck_kernel leaves, bit for bit
+        DraftStat ds;
+        ds.ml = Q.ml; ds.sx = Q.sx; ds.idx = Q.idx; ds.tag = kDraftStatTag ^ __float_as_uint(k);
+        static_cast<DraftStat *>(a.draft_stats_out)[r] = ds;
+    }
     if (!(Q.ml > neg_inf()) || !finite_pos(Zq) || !(Q.ml < -neg_inf())) {
         if (t0) {
             for (int m = 0; m < 3; ++m) {

@@ -25,6 +25,7 @@ def test_header_declares_the_expected_entry_points():
         "rrs_shard_sums", "rrs_shard_decide", "rrs_shard_draft", "rrs_shard_draft_finish",
         "spechub_draft_stats_bytes", "spechub_draft_sample_stats", "rrs_draft_sample_stats",
         "spechub_verify_tree_stats", "rrs_verify_tree_stats",
+        "mdsd_compare_draft_sample_stats", "mdsd_compare_verify_tree_stats",
         "spechub_workspace_bytes", "spechub_status_string", "spechub_abi_version"])
 
 

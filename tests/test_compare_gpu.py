@@ -97,6 +97,30 @@ def test_compare_calls(sh, V, dtype, paper):
         for k in SEQ_KEYS:
             np.testing.assert_array_equal(out[k], w[k], err_msg="walk %s %s" % (m, k))
 
+    # the same step with the draft statistics handed from the draft call to verification: one record per
+    # row serves the three methods; the per-method *_stats calls bit for bit, and the oracle
+    dall2 = sh.mdsd_compare_draft_sample_stats(tq, und, tree, Tt)
+    stats = dall2.pop("stats")
+    for m in METHODS:
+        for k in dall[m]:
+            np.testing.assert_array_equal(bits(dall2[m][k]), bits(dall[m][k]), err_msg="draft+stats %s %s" % (m, k))
+        if m == "spechub":
+            dsep = sh.spechub_draft_sample_stats(tq, und, tree, Tt)
+        else:
+            dsep = sh.rrs_draft_sample_stats(tq, und, tree, m == "rrsw", Tt)
+        np.testing.assert_array_equal(bits(dsep["stats"]), bits(stats), err_msg="records %s" % m)
+    vall2 = sh.mdsd_compare_verify_tree_stats(tp, tq, stats, toks, und, tree, Tt)
+    torch.cuda.synchronize()
+    for m in METHODS:
+        if m == "spechub":
+            vsep = sh.spechub_verify_tree_stats(tp, tq, stats, toks[m], und, tree, Tt)
+        else:
+            vsep = sh.rrs_verify_tree_stats(tp, tq, stats, toks[m], und, tree, m == "rrsw", Tt)
+        for k in NODE_KEYS + SEQ_KEYS:
+            np.testing.assert_array_equal(bits(vall2[m][k]), bits(vsep[k]), err_msg="verify+stats %s %s" % (m, k))
+        parity.check_verify(m, lp, lq, T, oracle_tokens[m], un, kind, parity.to_numpy(vall2[m]),
+                            label="compare-verify+stats")
+
     # without probability buffers: same decisions, tokens and walks
     lite = sh.mdsd_compare_verify_tree(tp, tq, toks, und, tree, Tt, probabilities=False)
     for m in METHODS:
