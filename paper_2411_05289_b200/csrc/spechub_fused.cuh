@@ -145,49 +145,53 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     float s1a, s2a, ra, s1b, s2b, rb, a1a, a1b, dna, dnb;
     unsigned diff = 0;
     auto pass_b = [&]() {
-    s1a = s2a = ra = s1b = s2b = rb = 0.f;
-    a1a = a1b = dna = dnb = 0.f;
+    // (packed as in lean_verify_kernel: the low lane of a pair takes the even ids of a vector, the high lane the
+    // odd ones; every sum keeps the association of the per-method kernels)
+    F2 s1 = f2_make(0.f, 0.f), s2 = s1, rr = s1, a1 = s1;
+    dna = dnb = 0.f;
+    const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ);
+    const F2 nrho2 = f2_make(-rho, -rho), ncrho2 = f2_make(-crho, -crho);
 #pragma unroll 2
     for (int vi = last_vi; vi >= lo; vi -= 32) {
-        float fp[8], fq[8];
         const uint4 rawp = vp[vi], rawq = vq[vi];
         if (STATS) diff |= (rawp.x ^ rawq.x) | (rawp.y ^ rawq.y) | (rawp.z ^ rawq.z) | (rawp.w ^ rawq.w);
-        unpack_bf16x8(rawp, fp);
-        unpack_bf16x8(rawq, fq);
-        float pp[8], qq[8];   // e_p, e_q (lean_terms: everything below is in units of 1 / Z_p)
+        const unsigned wps[4] = {rawp.x, rawp.y, rawp.z, rawp.w}, wqs[4] = {rawq.x, rawq.y, rawq.z, rawq.w};
+        float qw[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { pp[i] = lean_exp(fp[i], k, cP); qq[i] = lean_exp(fq[i], k, cQ); }
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            a1a += fmaxf(__fmaf_rn(-rho, qq[i], pp[i]), 0.f);
-            a1b += fmaxf(__fmaf_rn(-rho, qq[i + 1], pp[i + 1]), 0.f);
-        }
-        {
-            float qw[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) qw[i] = qq[i];
-            if (vi == wvec) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i == wel) qw[i] = 0.f;
+        for (int i = 0; i < 4; ++i) {
+            const F2 ep = f2_exp_word(wps[i], k2, ncp2);
+            F2 eq = f2_exp_word(wqs[i], k2, ncq2);
+            f2_get(eq, qw[2 * i], qw[2 * i + 1]);
+            F2 d = f2_fma(nrho2, eq, ep);              // Z_p (p - q)
+            F2 m = f2_max0(d);
+            a1 = f2_add(a1, m);                         // RRS / RRSw: over every id
+            if (vi == hubvec && i == (hubel >> 1)) {    // SpecHub's sums run over ids != a: that lane adds 0
+                float d0, d1, q0, q1;
+                f2_get(d, d0, d1);
+                f2_get(eq, q0, q1);
+                if (hubel & 1) { d1 = 0.f; q1 = 0.f; } else { d0 = 0.f; q0 = 0.f; }
+                d = f2_make(d0, d1);
+                eq = f2_make(q0, q1);
+                m = f2_max0(d);
             }
-            dna += (qw[0] + qw[1]) + (qw[2] + qw[3]);
-            dnb += (qw[4] + qw[5]) + (qw[6] + qw[7]);
+            const F2 t = f2_fma(ncrho2, eq, m);         // Z_p (max(p - q, 0) - c q)
+            const F2 w = f2_max0(t);
+            s1 = f2_add(s1, f2_sub(m, d));              // max(-d, 0) = max(d, 0) - d, exactly
+            s2 = f2_add(s2, f2_sub(w, t));
+            rr = f2_add(rr, w);
         }
-        if (vi == hubvec) {   // SpecHub's sums run over ids != a
+        if (vi == wvec) {   // RRSw's renormaliser leaves its x1 out
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                if (i == hubel) { pp[i] = 0.f; qq[i] = 0.f; }
+                if (i == wel) qw[i] = 0.f;
         }
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            float d, t;
-            lean_terms(pp[i], qq[i], rho, crho, d, t);
-            s1a += fmaxf(-d, 0.f); s2a += fmaxf(-t, 0.f); ra += fmaxf(t, 0.f);
-            lean_terms(pp[i + 1], qq[i + 1], rho, crho, d, t);
-            s1b += fmaxf(-d, 0.f); s2b += fmaxf(-t, 0.f); rb += fmaxf(t, 0.f);
-        }
+        dna += (qw[0] + qw[1]) + (qw[2] + qw[3]);
+        dnb += (qw[4] + qw[5]) + (qw[6] + qw[7]);
     }
+    f2_get(s1, s1a, s1b);
+    f2_get(s2, s2a, s2b);
+    f2_get(rr, ra, rb);
+    f2_get(a1, a1a, a1b);
     };
     pass_b();
     if (STATS && !__syncthreads_or(diff != 0)) {   // the target row is the draft row: Z_p = Z_q exactly
@@ -204,30 +208,27 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     const bool q1_zero = !(den > 0.f);
     const float A1g[2] = {A1, A1 * (q1_zero ? 0.f : 1.f / den)};
     const float A1grho[2] = {A1g[0] * rho, A1g[1] * rho};
-    float w0a = 0.f, w0b = 0.f, w1a = 0.f, w1b = 0.f;
+    float w0a, w0b, w1a, w1b;
+    {
+        F2 w0 = f2_make(0.f, 0.f), w1 = w0;
+        const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ), nrho2 = f2_make(-rho, -rho);
+        const F2 nsc0 = f2_make(-A1grho[0], -A1grho[0]), nsc1 = f2_make(-A1grho[1], -A1grho[1]);
 #pragma unroll 2
-    for (int vi = lo + lane; vi < hi; vi += 32) {
-        float fp[8], fq[8];
-        unpack_bf16x8(vp[vi], fp);
-        unpack_bf16x8(vq[vi], fq);
-        float sc[8];
+        for (int vi = lo + lane; vi < hi; vi += 32) {
+            const uint4 rawp = vp[vi], rawq = vq[vi];
+            const unsigned wps[4] = {rawp.x, rawp.y, rawp.z, rawp.w}, wqs[4] = {rawq.x, rawq.y, rawq.z, rawq.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) sc[i] = A1grho[1];
-        if (vi == wvec) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i == wel) sc[i] = 0.f;
+            for (int i = 0; i < 4; ++i) {
+                F2 nsc = nsc1;
+                if (vi == wvec && i == (wel >> 1)) nsc = (wel & 1) ? f2_make(-A1grho[1], 0.f) : f2_make(0.f, -A1grho[1]);
+                const F2 eq = f2_exp_word(wqs[i], k2, ncq2);
+                const F2 m = f2_max0(f2_fma(nrho2, eq, f2_exp_word(wps[i], k2, ncp2)));
+                w0 = f2_add(w0, f2_max0(f2_fma(nsc0, eq, m)));
+                w1 = f2_add(w1, f2_max0(f2_fma(nsc, eq, m)));
+            }
         }
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            const float p0 = lean_exp(fp[i], k, cP), q0 = lean_exp(fq[i], k, cQ);
-            const float p1 = lean_exp(fp[i + 1], k, cP), q1 = lean_exp(fq[i + 1], k, cQ);
-            float d, t;
-            lean_terms(p0, q0, rho, A1grho[0], d, t); w0a += fmaxf(t, 0.f);
-            lean_terms(p1, q1, rho, A1grho[0], d, t); w0b += fmaxf(t, 0.f);
-            lean_terms(p0, q0, rho, sc[i], d, t); w1a += fmaxf(t, 0.f);
-            lean_terms(p1, q1, rho, sc[i + 1], d, t); w1b += fmaxf(t, 0.f);
-        }
+        f2_get(w0, w0a, w0b);
+        f2_get(w1, w1a, w1b);
     }
     float accC[2] = {w0a + w0b, w1a + w1b};
     lean_block_sums<2, 5>(accC, sh);   // per-warp W2 stay in sh.acc[5], sh.acc[6]
