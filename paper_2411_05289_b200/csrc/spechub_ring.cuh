@@ -52,10 +52,10 @@ __device__ __forceinline__ void ring_issue(WarpRing &R) {
     const uint32_t bar = R.bars + 8u * st, dst = R.data + st * kRingStageBytes;
     const bool both = !(R.p_first && R.ipass == 0);
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(both ? 2u * bytes : bytes) : "memory");
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(R.vp + R.iv0), "r"(bytes), "r"(bar) : "memory");
     if (both)
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(dst + kRingChunkVecs * 16), "l"(R.vq + R.iv0), "r"(bytes), "r"(bar) : "memory");
     // the chunk after this one: the next of this pass, or the first of the next pass
     if (--R.ileft > 0) R.iv0 += R.istep;
