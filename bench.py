@@ -625,7 +625,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": dict(config_dict(cfg, args.layout, world),
                            draft_stats=("the draft call hands max / argmax / sum of each draft row to the verification "
-                                        "call (*_stats entry points): verification's first pass reads the target row only"
+                                        "call (*_stats entry points), written and read inside every timed step: verification's first pass "
+                                        "reads the target row only"
                                         if hand_over else "off: plain entry points")),
             "value_note": "each node is counted once per method (SpecHub, RRS, RRSw run one after another on the "
                           "same inputs): node-method verifications; SpecHub alone is breakdown.spechub_only_step",
