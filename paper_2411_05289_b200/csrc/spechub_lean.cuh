@@ -253,7 +253,6 @@ __device__ __forceinline__ void lean_pass_a_deep(const uint4 *rp, int lo, int hi
 }
 
 // Pass A over both rows with the vectors coming from the warp's ring (the first pass of its stream, forwards).
-template <bool BOTH>
 __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k, LeanAcc &P, LeanAcc &Q) {
     P.m2 = 0xff80ff80u; P.s = 0.f; P.c = 0.f;
     Q.m2 = 0xff80ff80u; Q.s = 0.f; Q.c = 0.f;
@@ -274,15 +273,13 @@ __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k,
                     if (m0 > neg_inf()) { P.c = shift_of(m0, k); break; }
                 }
             }
-            if (BOTH) {
-                m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
-                if (m0 > neg_inf()) Q.c = shift_of(m0, k);
-                else {
-                    for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
-                        const uint4 b2 = R.vq[vr];
-                        m0 = bf2_hmax(bf2max(bf2max(b2.x, b2.y), bf2max(b2.z, b2.w)));
-                        if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
-                    }
+            m0 = bf2_hmax(bf2max(bf2max(b.x, b.y), bf2max(b.z, b.w)));
+            if (m0 > neg_inf()) Q.c = shift_of(m0, k);
+            else {
+                for (int vr = vi0 + 32; vr < R.hi; vr += 32) {
+                    const uint4 b2 = R.vq[vr];
+                    m0 = bf2_hmax(bf2max(bf2max(b2.x, b2.y), bf2max(b2.z, b2.w)));
+                    if (m0 > neg_inf()) { Q.c = shift_of(m0, k); break; }
                 }
             }
         }
@@ -298,7 +295,7 @@ __device__ __forceinline__ void lean_pass_a_ring(WarpRing &R, int lane, float k,
             if (j == kRingCh - 1) ring_release(R, lane);
             if (v0 + j * 32 < R.hi) {
                 lean_push(P, x, k);
-                if (BOTH) lean_push(Q, y, k);
+                lean_push(Q, y, k);
             }
         }
     }
@@ -940,8 +937,8 @@ __device__ __forceinline__ void lean_terms(float ep, float eq, float rho, float 
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
-// RING (RRS and RRSw, one CTA per row): the three passes take their vectors from per-warp rings of bulk
-// copies (spechub_ring.cuh; THREADS / 32 * kRingWarpBytes of dynamic shared memory) instead of loading
+// RING (RRS and RRSw, one CTA per row): the passes over both rows take their vectors from per-warp rings of
+// bulk copies (spechub_ring.cuh; THREADS / 32 * kRingWarpBytes of dynamic shared memory) instead of loading
 // them from global memory into registers.  Measured on V = 128256, 7936 rows: RRS 1.89 -> 1.72 ms, RRSw
 // 1.99 -> 1.86 ms; SpecHub's two passes gain nothing from it (1.38 -> 1.38 .. 1.44 ms: the bookkeeping of
 // the ring costs the issue slots that its pass B is short of), so SpecHub keeps the register-fed loops.
@@ -985,9 +982,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
 
     // the row's stream: pass A forwards, pass B backwards, (RRS, RRSw) pass C forwards
     WarpRing R;
-    if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, STATS, lane);
+    // (from draft statistics pass A reads the target row only, with plain loads; the ring then feeds B and C,
+    // whose first chunks are on their way while pass A runs: 1.54 -> 1.53 ms against a ring-fed pass A)
+    if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, STATS ? 2 : 3, STATS ? 1u : 2u, lane);
     LeanAcc tp, tq;
-    if (RING) lean_pass_a_ring<!STATS>(R, lane, k, tp, tq);
+    if (RING && !STATS) lean_pass_a_ring(R, lane, k, tp, tq);
     else if (STATS) lean_pass_a_deep(vp, lo, hi, lane, k, tp);
     else if (leaf) lean_pass_a<false>(vp, vq, lo, hi, lane, k, tp, tq);
     else lean_pass_a<true, METHOD == kRRS>(vp, vq, lo, hi, lane, k, tp, tq);

@@ -41,7 +41,6 @@ struct WarpRing {
     int issued;      // chunks requested so far (the same in every lane; lane 0 issues)
     int ipass, ileft, iv0, istep;   // lane 0: the next chunk to request (its pass, chunks left in it, first vector, stride)
     unsigned back;   // bit i: pass i runs from the top of the range down
-    bool p_first;    // the first pass reads the target row only
     bool timed_out;
 };
 
@@ -50,13 +49,11 @@ __device__ __forceinline__ void ring_issue(WarpRing &R) {
     const uint32_t bytes = static_cast<uint32_t>(min(kRingChunkVecs, R.hi - R.iv0)) * 16u;
     const uint32_t st = static_cast<uint32_t>(R.issued) & (kRingStages - 1);
     const uint32_t bar = R.bars + 8u * st, dst = R.data + st * kRingStageBytes;
-    const bool both = !(R.p_first && R.ipass == 0);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(both ? 2u * bytes : bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2u * bytes) : "memory");
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(R.vp + R.iv0), "r"(bytes), "r"(bar) : "memory");
-    if (both)
-        asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst + kRingChunkVecs * 16), "l"(R.vq + R.iv0), "r"(bytes), "r"(bar) : "memory");
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst + kRingChunkVecs * 16), "l"(R.vq + R.iv0), "r"(bytes), "r"(bar) : "memory");
     // the chunk after this one: the next of this pass, or the first of the next pass
     if (--R.ileft > 0) R.iv0 += R.istep;
     else {
@@ -69,15 +66,14 @@ __device__ __forceinline__ void ring_issue(WarpRing &R) {
 }
 
 // All lanes of the warp.  `data` / `bars`: this warp's kRingWarpBytes (16-byte aligned) and its kRingStages
-// mbarriers in shared memory.  `passes` passes over [lo, hi); bit i of `back` makes pass i run backwards;
-// p_first: the first pass brings the target row only (the draft half of its stages is not written).
+// mbarriers in shared memory.  `passes` passes over [lo, hi); bit i of `back` makes pass i run backwards.
 __device__ __forceinline__ void ring_begin(WarpRing &R, void *data, uint64_t *bars, const uint4 *vp, const uint4 *vq,
-                                           int lo, int hi, int passes, unsigned back, bool p_first, int lane) {
+                                           int lo, int hi, int passes, unsigned back, int lane) {
     R.data = ring_saddr(data); R.bars = ring_saddr(bars);
     R.vp = vp; R.vq = vq; R.lo = lo; R.hi = hi;
     R.nc = hi > lo ? (hi - lo + kRingChunkVecs - 1) / kRingChunkVecs : 0;
     R.ng = passes * R.nc;
-    R.g = 0; R.issued = 0; R.back = back; R.p_first = p_first; R.timed_out = false;
+    R.g = 0; R.issued = 0; R.back = back; R.timed_out = false;
     R.ipass = 0; R.ileft = R.nc;
     R.istep = (back & 1u) ? -kRingChunkVecs : kRingChunkVecs;
     R.iv0 = (back & 1u) ? lo + (R.nc - 1) * kRingChunkVecs : lo;
