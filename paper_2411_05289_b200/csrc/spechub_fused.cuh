@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         for (int i = 0; i < 4; ++i) {
             const F2 ep = f2_exp_word(wps[i], k2, ncp2);
             F2 eq = f2_exp_word(wqs[i], k2, ncq2);
-            f2_get(eq, qw[2 * i], qw[2 * i + 1]);
+            if (!STATS) f2_get(eq, qw[2 * i], qw[2 * i + 1]);
             F2 d = f2_fma(nrho2, eq, ep);              // Z_p (p - q)
             F2 m = f2_max0(d);
             a1 = f2_add(a1, m);                         // RRS / RRSw: over every id
@@ -180,13 +180,15 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
             s2 = f2_add(s2, f2_sub(w, t));
             rr = f2_add(rr, w);
         }
-        if (vi == wvec) {   // RRSw's renormaliser leaves its x1 out
+        if (!STATS) {   // RRSw's renormaliser leaves its x1 out (from draft statistics: sum_without, below)
+            if (vi == wvec) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i == wel) qw[i] = 0.f;
+                for (int i = 0; i < 8; ++i)
+                    if (i == wel) qw[i] = 0.f;
+            }
+            dna += (qw[0] + qw[1]) + (qw[2] + qw[3]);
+            dnb += (qw[4] + qw[5]) + (qw[6] + qw[7]);
         }
-        dna += (qw[0] + qw[1]) + (qw[2] + qw[3]);
-        dnb += (qw[4] + qw[5]) + (qw[6] + qw[7]);
     }
     f2_get(s1, s1a, s1b);
     f2_get(s2, s2a, s2b);
@@ -200,6 +202,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
     }
     float accB[5] = {s1a + s1b, s2a + s2b, ra + rb, a1a + a1b, dna + dnb};
     lean_block_sums<5, 0>(accB, sh);   // per-warp R stays in sh.acc[2]
+    if (STATS) accB[4] = wx1 >= 0 ? sum_without(Q, rowq, wx1, k) : 0.f;
     const float Rraw = accB[2];
     const float S1 = accB[0] * invZp, S2 = degenerate ? qa : accB[1] * invZp, R = Rraw * invZp;
     const float A1 = accB[3] * invZp, den = accB[4] * invZq;

@@ -934,6 +934,14 @@ __device__ __forceinline__ void lean_terms(float ep, float eq, float rho, float 
     t = __fmaf_rn(-srho, eq, fmaxf(d, 0.f));
 }
 
+// Sum of a row's exponentials outside id x, from the row's (maximum, argmax, sum without the argmax): RRSw's
+// renormaliser 1 - q(x1) times Z_q without a pass over the row.  The argmax is left out of st.sx already; any
+// other id holds at most half of the mass, so subtracting its own term costs at most one bit.
+__device__ __forceinline__ float sum_without(const RowStat &st, const __nv_bfloat16 *row, int x, float k) {
+    if (x == st.idx) return st.sx;
+    return __fsub_rn(__fadd_rn(st.sx, st.own), lean_exp(load_one<__nv_bfloat16>(row, x), k, st.C));
+}
+
 // ------------------------------------------------------------------------------------------------
 // Verification (SpecHub: Algorithm 3; RRS / RRSw: Algorithm 1) and leaf draws.
 // ------------------------------------------------------------------------------------------------
@@ -1202,7 +1210,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             }
             // pass B: A1 = sum max(p - q, 0); RRSw also sums q outside x1 directly
             const int x1vec = x1 >> 3, x1el = x1 & 7;
-            float dna, dnb;
+            float dna = 0.f, dnb = 0.f;
             F2 a1;   // (packed: low lane = even ids of a vector, high lane = odd ids)
             const F2 k2 = f2_make(k, k), ncq2 = f2_make(-cQ, -cQ);
             F2 ncp2, nrho2;
@@ -1218,7 +1226,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
                     eq[i] = f2_exp_word(wqs[i], k2, ncq2);
                     a1 = f2_add(a1, f2_max0(f2_fma(nrho2, eq[i], f2_exp_word(wps[i], k2, ncp2))));
                 }
-                if (METHOD == kRRSw) {
+                if (METHOD == kRRSw && !STATS) {   // (from draft statistics: sum_without, below)
                     float qq[8];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) f2_get(eq[i], qq[2 * i], qq[2 * i + 1]);
@@ -1270,6 +1278,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             float acc[2] = {a1a + a1b, dna + dnb};
             float part2[2][CS];
             lean_row_sums<CS, 2, 0>(acc, part2, sh);  // [2]
+            if (STATS && METHOD == kRRSw) acc[1] = sum_without(Q, rowq, x1, k);
             const float A1 = acc[0] * invZp, den = acc[1] * invZq;   // the sums are of exponentials
             const bool q1_zero = (METHOD == kRRSw) && !(den > 0.f);
             const float gq = (METHOD == kRRSw) ? (q1_zero ? 0.f : 1.f / den) : 1.f;
