@@ -363,17 +363,19 @@ def main():
     # instead of twice; off = the plain entry points.
     hand_over = args.draft_stats == "on"
 
-    def do_draft(m, tq, un):
+    def do_draft(m, tq, un, ho=None):
+        ho = hand_over if ho is None else ho
         if m == "spechub":
-            return (sh.spechub_draft_sample_stats if hand_over else sh.spechub_draft_sample)(tq, un, tree, cfg.temperature)
-        return (sh.rrs_draft_sample_stats if hand_over else sh.rrs_draft_sample)(tq, un, tree, m == "rrsw", cfg.temperature)
+            return (sh.spechub_draft_sample_stats if ho else sh.spechub_draft_sample)(tq, un, tree, cfg.temperature)
+        return (sh.rrs_draft_sample_stats if ho else sh.rrs_draft_sample)(tq, un, tree, m == "rrsw", cfg.temperature)
 
-    def do_verify(m, tp, tq, d, un, out):
+    def do_verify(m, tp, tq, d, un, out, ho=None):
+        ho = hand_over if ho is None else ho
         if m == "spechub":
-            if hand_over:
+            if ho:
                 return sh.spechub_verify_tree_stats(tp, tq, d["stats"], d["tokens"], un, tree, cfg.temperature, out=out)
             return sh.spechub_verify_tree(tp, tq, d["tokens"], un, tree, cfg.temperature, out=out)
-        if hand_over:
+        if ho:
             return sh.rrs_verify_tree_stats(tp, tq, d["stats"], d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=out)
         return sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, m == "rrsw", cfg.temperature, out=out)
 
@@ -417,6 +419,26 @@ def main():
     # per API call: mean device time of its kernels (a verify call = verification kernel + walk kernel)
     call_ms = {k: float(np.mean([a.elapsed_time(b) for a, b in v])) for k, v in ev_pairs.items()}
     verify_ms = call_ms["spechub_verify_tree"]
+
+    # ---- extra: the same step through the other set of entry points (plain if the timed step hands the draft
+    # statistics over, and the other way round) ----
+    def other_step():
+        tp_, tq_, un_ = copies[turn[0] % len(copies)]
+        turn[0] += 1
+        for m in METHODS:
+            d = do_draft(m, tq_, un_, not hand_over)
+            do_verify(m, tp_, tq_, d, un_, outs[m], not hand_over)
+
+    for _ in range(3):
+        other_step()
+    barrier()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    o0.record(stream)
+    for _ in range(args.steps):
+        other_step()
+    o1.record(stream)
+    barrier()
+    other_ms = o0.elapsed_time(o1) / args.steps
 
     # ---- extra: SpecHub verification when the caller asks for decisions and tokens only ----
     d0 = sh.spechub_draft_sample(tq, un, tree, cfg.temperature)
@@ -666,6 +688,11 @@ def main():
                     "ms_per_launch": lite_ms, "nodes_per_s": B * N / (lite_ms * 1e-3),
                     "note": "beta / rate not requested: rows whose first test accepts skip pass B; "
                             "not part of `value`"},
+                "step_through_the_other_entry_points": {
+                    "ms_per_step": other_ms, "nodes_per_s": len(METHODS) * B * N / (other_ms * 1e-3),
+                    "note": ("the plain entry points (no hand-over of draft statistics)" if hand_over else
+                             "the _stats entry points (draft statistics handed to verification)")
+                            + "; this rank only; not part of `value`"},
                 "step_as_cuda_graph": {
                     "ms_per_step": graph_ms,
                     "nodes_per_s": (len(METHODS) * B * N / (graph_ms * 1e-3)) if graph_ms else None,
