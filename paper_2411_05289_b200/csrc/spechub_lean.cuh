@@ -144,6 +144,14 @@ __device__ __forceinline__ F2 f2_exp_word(unsigned w, F2 k2, F2 nc2) {
     return f2_make(ex2(x0), ex2(x1));
 }
 
+// a 16-byte load with an L2 eviction policy (createpolicy)
+__device__ __forceinline__ uint4 ld_l2_hint(const uint4 *p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+
 struct LeanAcc {  // one thread's pass-A state for one row
     unsigned m2;  // packed running maximum
     float c;      // exponent reference (k * some logit of this thread, or 0)
@@ -216,13 +224,6 @@ __device__ __forceinline__ void lean_pass_a(const uint4 *rp, const uint4 *rq, in
 
 // Pass A over one row with four vectors per lane in flight: the next four are requested before the current
 // four are consumed.  Same vectors in the same order as lean_pass_a<false>, so the same sums.
-// a 16-byte load with an L2 eviction policy (createpolicy)
-__device__ __forceinline__ uint4 ld_l2_hint(const uint4 *p, uint64_t pol) {
-    uint4 v;
-    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
-    return v;
-}
 __device__ __forceinline__ void lean_pass_a_deep(const uint4 *rp, int lo, int hi, int lane, float k, LeanAcc &P) {
     uint64_t pol;   // the row is read again by pass B: L2 is asked to keep it
     asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -1119,12 +1120,14 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
             };
             {
                 // software pipeline: the next vector pair is in registers before this one is consumed.
-                // From draft statistics this is the last use of both rows: the loads tell L2 to let these
-                // lines go first (and pass A told it to keep the target row's), 1.07 -> 1.02 ms on
-                // V = 128256; the kernel that reads both rows twice loses with such hints.
+                // This is the last use of both rows: the loads tell L2 to let these lines go first (one
+                // CTA per row: 1.38 -> 1.30 ms on V = 128256; from draft statistics, where pass A also told
+                // L2 to keep the target row's lines, 1.07 -> 1.02 ms.  Keep-hints on pass A of the kernel
+                // that reads both rows twice cost it 7-13 %).
                 uint64_t polf = 0;
-                if (STATS) asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(polf));
-                auto ldb = [&](const uint4 *ptr) { return STATS ? ld_l2_hint(ptr, polf) : *ptr; };
+                constexpr bool kHintB = STATS || CS == 1;
+                if (kHintB) asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(polf));
+                auto ldb = [&](const uint4 *ptr) { return kHintB ? ld_l2_hint(ptr, polf) : *ptr; };
                 uint4 np = make_uint4(0, 0, 0, 0), nq = np;
                 if (last_vi >= lo) { np = ldb(vp + last_vi); nq = ldb(vq + last_vi); }
 #pragma unroll 1
