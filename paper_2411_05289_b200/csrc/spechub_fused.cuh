@@ -216,9 +216,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) fused_verify_kernel(F
         F2 w0 = f2_make(0.f, 0.f), w1 = w0;
         const F2 k2 = f2_make(k, k), ncp2 = f2_make(-cP, -cP), ncq2 = f2_make(-cQ, -cQ), nrho2 = f2_make(-rho, -rho);
         const F2 nsc0 = f2_make(-A1grho[0], -A1grho[0]), nsc1 = f2_make(-A1grho[1], -A1grho[1]);
+        uint64_t polf;   // the rows' last use: L2 may let these lines go first
+        asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(polf));
 #pragma unroll 2
         for (int vi = lo + lane; vi < hi; vi += 32) {
-            const uint4 rawp = vp[vi], rawq = vq[vi];
+            const uint4 rawp = ld_l2_hint(vp + vi, polf), rawq = ld_l2_hint(vq + vi, polf);
             const unsigned wps[4] = {rawp.x, rawp.y, rawp.z, rawp.w}, wqs[4] = {rawq.x, rawq.y, rawq.z, rawq.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
