@@ -121,9 +121,9 @@ int launch_lean_leaf(const RowArgs &a, const NodeOutPtrs *outs, int n_out, unsig
 }
 
 // One CTA per row, the passes fed by per-warp rings of bulk copies (spechub_ring.cuh).
-template <int METHOD, bool STATS>
+template <int METHOD>
 int launch_lean_verify_ring(const RowArgs &a, unsigned rows, cudaStream_t s) {
-    auto kern = lean_verify_kernel<METHOD, kLeanThreads, 1, true, STATS>;
+    auto kern = lean_verify_kernel<METHOD, kLeanThreads, 1, true>;
     constexpr int smem = kLeanThreads / 32 * kRingWarpBytes;
     static bool configured[kMaxDevices] = {};
     int dev = -1;
@@ -151,16 +151,14 @@ int launch_lean_verify(int method, int cs, const RowArgs &a, unsigned rows, cuda
         if (lrc != SPECHUB_OK) return lrc;
     }
     if (cs == 0 && a.draft_stats_in) {   // the draft row's statistics come from the draft step
-        if (method == kSpecHub) {
-            lean_verify_kernel<kSpecHub, kLeanThreads, 1, false, true><<<rows, kLeanThreads, 0, s>>>(a);
-            return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
-        }
-        if (method == kRRS) return launch_lean_verify_ring<kRRS, true>(a, rows, s);
-        return launch_lean_verify_ring<kRRSw, true>(a, rows, s);
+        if (method == kSpecHub) lean_verify_kernel<kSpecHub, kLeanThreads, 1, false, true><<<rows, kLeanThreads, 0, s>>>(a);
+        else if (method == kRRS) lean_verify_kernel<kRRS, kLeanThreads, 1, false, true><<<rows, kLeanThreads, 0, s>>>(a);
+        else lean_verify_kernel<kRRSw, kLeanThreads, 1, false, true><<<rows, kLeanThreads, 0, s>>>(a);
+        return cudaGetLastError() == cudaSuccess ? SPECHUB_OK : SPECHUB_ERR_LAUNCH;
     }
     if (cs == 1 || method == kSpecHub) return launch_lean_verify_cs<1>(method, a, rows, s);
-    if (method == kRRS) return launch_lean_verify_ring<kRRS, false>(a, rows, s);
-    return launch_lean_verify_ring<kRRSw, false>(a, rows, s);
+    if (method == kRRS) return launch_lean_verify_ring<kRRS>(a, rows, s);
+    return launch_lean_verify_ring<kRRSw>(a, rows, s);
 }
 int launch_lean_draft(int method, int cs, const RowArgs &a, unsigned rows, cudaStream_t s) {
     if (cs == 4) return launch_group(lean_draft_kernel<kLeanThreads, 4>, 4, rows, s, a, method);
