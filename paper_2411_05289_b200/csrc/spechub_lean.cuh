@@ -991,6 +991,19 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
     // a flagged row, the CTA that draws for a residual / leaf token.
     bool token_elsewhere = false;
 
+    if (STATS && threadIdx.x == THREADS - 1) {
+        // The draft row's record, fetched and checked by one thread before it starts on pass A: its two
+        // dependent look-ups (the record, then the draft logit at the recorded argmax) are off the path
+        // between pass A and pass B.  (Nothing else writes these fields; they are read after barriers.)
+        const DraftStat ds = static_cast<const DraftStat *>(a.draft_stats_in)[r];
+        bool ok = ds.tag == (kDraftStatTag ^ __float_as_uint(k));
+        // (a record of a row without a finite maximum or sum needs no look-up: the row is flagged
+        // SPECHUB_ST_NONFINITE below, as it is without the record)
+        if (ok && ds.ml > neg_inf() && ds.ml < pinf && finite_pos(ds.sx + 1.f))
+            ok = ds.idx >= 0 && ds.idx < a.vocab && load_one<__nv_bfloat16>(rowq, ds.idx) == ds.ml;
+        sh.stat_ok = ok;
+        sh.x_ml[1] = ds.ml; sh.x_sx[1] = ds.sx; sh.x_idx[1] = ok ? ds.idx : 0;
+    }
     // the row's stream: pass A forwards, pass B backwards, (RRS, RRSw) pass C forwards
     WarpRing R;
     if (RING) ring_begin(R, ring_mem + warp * kRingWarpBytes, ring_bars[warp], vp, vq, lo, hi, 3, 2u, lane);
@@ -1005,18 +1018,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) lean_verify_kernel(Ro
         else lean_reduce2<true>(tp, tq, vp, vq, lo, hi, k, sh, Ps, Qs);
         if (threadIdx.x == 0) {
             sh.x_ml[0] = Ps.ml; sh.x_sx[0] = Ps.sx; sh.x_idx[0] = Ps.idx;
-            if (STATS) {
-                const DraftStat ds = static_cast<const DraftStat *>(a.draft_stats_in)[r];
-                bool ok = ds.tag == (kDraftStatTag ^ __float_as_uint(k));
-                // (a record of a row without a finite maximum or sum needs no look-up: the row is flagged
-                // SPECHUB_ST_NONFINITE below, as it is without the record)
-                if (ok && ds.ml > neg_inf() && ds.ml < pinf && finite_pos(ds.sx + 1.f))
-                    ok = ds.idx >= 0 && ds.idx < a.vocab && load_one<__nv_bfloat16>(rowq, ds.idx) == ds.ml;
-                sh.stat_ok = ok;
-                sh.x_ml[1] = ds.ml; sh.x_sx[1] = ds.sx; sh.x_idx[1] = ok ? ds.idx : 0;
-            } else {
-                sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx;
-            }
+            if (!STATS) { sh.x_ml[1] = Qs.ml; sh.x_sx[1] = Qs.sx; sh.x_idx[1] = Qs.idx; }
         }
     }
     RowGroup<CS>::sync();  // [1] slices published
