@@ -42,11 +42,11 @@ METHODS = ("spechub", "rrs", "rrsw")
 # is of the default step (--draft-stats on, --verify-path default); any other path reports no traffic.
 TRAFFIC_PER_ROW = {
     ("spechub_draft_sample", "c4"): 275593472.0 / 992,
-    ("spechub_verify_tree", "c4"): 623461376.0 / 992,
+    ("spechub_verify_tree", "c4"): 624340992.0 / 992,
     ("rrs_draft_sample[rrs]", "c4"): 281195008.0 / 992,
-    ("rrs_verify_tree[rrs]", "c4"): 981361664.0 / 992,
+    ("rrs_verify_tree[rrs]", "c4"): 977194496.0 / 992,
     ("rrs_draft_sample[rrsw]", "c4"): 279507712.0 / 992,
-    ("rrs_verify_tree[rrsw]", "c4"): 1006009344.0 / 992,
+    ("rrs_verify_tree[rrsw]", "c4"): 1008760320.0 / 992,
 }
 
 
