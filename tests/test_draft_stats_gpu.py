@@ -145,3 +145,25 @@ def test_records_are_reusable_and_the_buffer_is_checked(sh):
         assert torch.equal(a[k], b[k]), k
     with pytest.raises(ValueError):
         verify(sh, "spechub", tp, tq, d, un, tree, stats=d["stats"][:8])
+
+
+def test_more_than_two_drafts_neither_write_nor_read_records(sh):
+    """k = 3 (RRS / RRSw only): the draft kernels of that path keep no statistics and its verification
+    kernels take none; the *_stats calls are the plain calls."""
+    rng = np.random.default_rng(21)
+    tree = sh.Tree.kary(3, 3)
+    B, N, V = 3, tree.nodes_of_complete_tree(), 16384
+    lp = rng.normal(0, 2.0, (B, N, V)).astype(np.float32)
+    lq = lp + rng.normal(0, 1.0, (B, N, V)).astype(np.float32)
+    tp, tq = workloads.to_device(lp, "bf16", "cuda"), workloads.to_device(lq, "bf16", "cuda")
+    un = torch.from_numpy(rng.integers(0, 1 << 24, (B, N, 7)).astype(np.float32) * np.float32(2.0 ** -24)).cuda()
+    for wo in (False, True):
+        d = sh.rrs_draft_sample_stats(tq, un, tree, wo)
+        plain_d = sh.rrs_draft_sample(tq, un, tree, wo)
+        assert int(d["stats"].abs().sum()) == 0
+        assert torch.equal(d["tokens"], plain_d["tokens"])
+        a = sh.rrs_verify_tree(tp, tq, d["tokens"], un, tree, wo)
+        b = sh.rrs_verify_tree_stats(tp, tq, d["stats"], d["tokens"], un, tree, wo)
+        torch.cuda.synchronize()
+        for k in a:
+            assert torch.equal(a[k], b[k]), (wo, k)
