@@ -25,8 +25,10 @@
  *     at any data pointer.
  *   - Per-row problems found on the device are reported as bits in the row's
  *     `status` word and give the documented fallback output; kernels never
- *     trap and wait only on hardware barriers (and, where stated, on the
- *     hardware's tensor-memory allocator).
+ *     trap and wait only on hardware barriers, on the completion of bulk
+ *     copies they issued themselves (a bounded wait: SPECHUB_ST_INTERNAL if
+ *     it runs out) and, where stated, on the hardware's tensor-memory
+ *     allocator.
  *   - Layout: logits are [batch][nodes][vocab] with element strides
  *     `stride_seq`, `stride_node` (rows are contiguous in the vocabulary).
  *     Rows that start on a 16-byte boundary are read with 128-bit loads; other
